@@ -1,0 +1,230 @@
+"""Plain CPU oracle for the SnapKV prompt KV-cache compression step.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, obviously-correct statement of
+what the compression step computes, written from the paper (Sec. 4, Eq. 1-2 and
+Listing 1) in fp64.  It shares no code with the CUDA path and must never be
+imported by the product package; only the tests, the smoke check and the
+benchmark's CPU-baseline leg call it.
+
+Notation (paper, Sec. 4): L = L_prompt, W = L_obs (observation window), n = L - W =
+L_prefix, k = budget - W selected prefix rows, r = pool_kernel // 2.
+
+Inputs are bf16 tensors passed as numpy uint16 bit patterns so that no precision
+is lost or invented on the way in and the gathered rows can be compared bit for
+bit.  Shapes follow Listing 1: q_obs [B, Hq, W, d] (the last W prompt queries),
+k and v [B, Hkv, L, d].  With grouped-query attention query head h reads KV head
+h // (Hq // Hkv).
+
+Readings of points the paper leaves open (all listed again in the design notes):
+  * logits are q.k / sqrt(d), the mask is purely causal: window row i sees keys
+    j <= n + i;
+  * the softmax normaliser runs over every visible key (prefix and window), the
+    slice to the prefix happens after normalisation (Listing 1 slices after
+    compute_attn);
+  * Eq. 1's sum runs over the W window rows (Listing 1's .sum over the window axis);
+  * k = budget - W (Listing 1), not floor(p * L_prefix);
+  * average pooling divides by pool_kernel everywhere (zero padding counted);
+    max pooling ignores positions outside [0, n);
+  * ties in the top-k go to the lower position; indices are emitted ascending;
+  * budget >= L is the identity.
+
+Every function here is pinned by tests that do not go through this file's own
+formulas (closed forms, invariants, library routines, brute force): see
+tests/test_oracle_*.py.  Nothing is "parity unpinned".
+"""
+from __future__ import annotations
+
+import math
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+POOL_MAX = 0
+POOL_AVG = 1
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Widen bf16 bit patterns (uint16) to fp64 exactly.
+
+    A bf16 number is the upper half of an IEEE fp32 number, so placing the 16 bits
+    in the high half of a 32-bit word and reading it as fp32 is exact.
+    """
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    with np.errstate(invalid="ignore"):  # signalling-NaN patterns are quieted by the cast
+        return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def window_logits(q_head: np.ndarray, k_head: np.ndarray) -> np.ndarray:
+    """s[i, j] = q_i . k_j / sqrt(d) for one head (Listing 1, compute_attn).
+
+    q_head: [W, d] fp64, k_head: [L, d] fp64 -> [W, L] fp64.
+    """
+    d = q_head.shape[-1]
+    return (q_head @ k_head.T) / math.sqrt(d)
+
+
+def window_softmax(s: np.ndarray) -> np.ndarray:
+    """Causally masked, softmax-normalised attention of the window rows (Sec. 4,
+    "softmax-normalized attention features").
+
+    s: [W, L] logits.  Window row i is prompt position n + i and sees keys
+    j <= n + i.  Returns p [W, L] with zeros at masked positions; every row sums
+    to one over its visible keys.
+    """
+    W, L = s.shape
+    n = L - W
+    j = np.arange(L)[None, :]
+    i = np.arange(W)[:, None]
+    visible = j <= (n + i)
+    masked = np.where(visible, s, -np.inf)
+    m = masked.max(axis=1, keepdims=True)
+    e = np.where(visible, np.exp(masked - m), 0.0)
+    return e / e.sum(axis=1, keepdims=True)
+
+
+def vote_from_probs(p: np.ndarray) -> np.ndarray:
+    """Eq. 1: C[j] = sum over the W window rows of p[i, j], prefix columns only."""
+    W, L = p.shape
+    n = L - W
+    return p[:, :n].sum(axis=0)
+
+
+def window_votes(q_head: np.ndarray, k_head: np.ndarray) -> np.ndarray:
+    """Steps score -> softmax -> vote for one head: [W,d],[L,d] -> [n]."""
+    return vote_from_probs(window_softmax(window_logits(q_head, k_head)))
+
+
+def pool1d(vote: np.ndarray, pool_kernel: int, pool_type: int) -> np.ndarray:
+    """Listing 1's pool1d(kernel_size, padding=kernel_size//2, stride=1) on one row.
+
+    max: maximum over the in-range neighbours |t| <= r.
+    avg: sum over the in-range neighbours divided by pool_kernel (zero padding
+    counted in the divisor).
+    """
+    if pool_kernel < 1 or pool_kernel % 2 == 0:
+        raise ValueError("pool_kernel must be odd and >= 1")
+    if pool_type not in (POOL_MAX, POOL_AVG):
+        raise ValueError("pool_type must be POOL_MAX or POOL_AVG")
+    n = vote.shape[0]
+    r = pool_kernel // 2
+    # Pad r positions on both sides with the neutral element, then look at the
+    # pool_kernel shifted copies: copy t holds vote[j + t - r] at position j.
+    fill = -np.inf if pool_type == POOL_MAX else 0.0
+    padded = np.concatenate([np.full(r, fill), vote.astype(np.float64), np.full(r, fill)])
+    shifted = np.stack([padded[t:t + n] for t in range(pool_kernel)])
+    if pool_type == POOL_MAX:
+        return shifted.max(axis=0)
+    return shifted.sum(axis=0) / pool_kernel
+
+
+def topk_positions(pooled: np.ndarray, k: int) -> np.ndarray:
+    """Eq. 2: the k positions of largest pooled vote, ties to the lower position,
+    returned in ascending position order (int64)."""
+    n = pooled.shape[0]
+    if not 0 <= k <= n:
+        raise ValueError("k out of range")
+    order = np.argsort(-pooled, kind="stable")  # value descending, index ascending
+    return np.sort(order[:k])
+
+
+def kv_head_of(h: int, Hq: int, Hkv: int) -> int:
+    """Consecutive query heads share one KV head."""
+    return h // (Hq // Hkv)
+
+
+def _check_shapes(q_obs, k, v):
+    B, Hq, W, d = q_obs.shape
+    Bk, Hkv, L, dk = k.shape
+    if v.shape != k.shape or Bk != B or dk != d:
+        raise ValueError("inconsistent shapes")
+    if Hq % Hkv != 0:
+        raise ValueError("Hq must be a multiple of Hkv")
+    if W > L:
+        raise ValueError("window longer than the prompt")
+    return B, Hq, Hkv, L, d, W
+
+
+def votes(q_obs: np.ndarray, k: np.ndarray, workers: int = 1) -> np.ndarray:
+    """Votes for every (batch, query head): bf16 bits in, fp64 [B, Hq, n] out."""
+    B, Hq, W, d = q_obs.shape
+    _, Hkv, L, _ = k.shape
+    n = L - W
+    out = np.empty((B, Hq, n), dtype=np.float64)
+
+    def unit(bc):
+        b, c = bc
+        kf = bf16_bits_to_f64(k[b, c])
+        g = Hq // Hkv
+        for h in range(c * g, (c + 1) * g):
+            out[b, h] = window_votes(bf16_bits_to_f64(q_obs[b, h]), kf)
+
+    units = [(b, c) for b in range(B) for c in range(Hkv)]
+    if workers > 1:
+        with ThreadPoolExecutor(max_workers=workers) as ex:
+            list(ex.map(unit, units))
+    else:
+        for u in units:
+            unit(u)
+    return out
+
+
+def compress(q_obs: np.ndarray, k: np.ndarray, v: np.ndarray, pool_kernel: int,
+             pool_type: int, budget: int, workers: int = 1, heads=None):
+    """The whole step (Listing 1) on bf16 bit patterns.
+
+    Returns a dict with
+      out_k, out_v : uint16 [B, Hq, rows, d], rows = min(budget, L)
+      out_idx      : int64  [B, Hq, rows - W] ascending prefix positions
+      vote, pooled : fp64   [B, Hq, n] (None on the identity path)
+    `heads` optionally restricts the work to a list of (b, h) pairs (other heads
+    are left zero) so that sampled checks at large sizes stay affordable.
+    """
+    B, Hq, Hkv, L, d, W = _check_shapes(q_obs, k, v)
+    if budget <= W:
+        raise ValueError("budget must exceed the window")
+    n = L - W
+    g = Hq // Hkv
+    if budget >= L:  # Listing 1's early return: nothing is dropped
+        kv_of = [kv_head_of(h, Hq, Hkv) for h in range(Hq)]
+        return {
+            "out_k": np.ascontiguousarray(k[:, kv_of]),
+            "out_v": np.ascontiguousarray(v[:, kv_of]),
+            "out_idx": np.broadcast_to(np.arange(n, dtype=np.int64), (B, Hq, n)).copy(),
+            "vote": None,
+            "pooled": None,
+        }
+    ksel = budget - W
+    out_k = np.zeros((B, Hq, budget, d), dtype=np.uint16)
+    out_v = np.zeros((B, Hq, budget, d), dtype=np.uint16)
+    out_idx = np.zeros((B, Hq, ksel), dtype=np.int64)
+    vote = np.zeros((B, Hq, n), dtype=np.float64)
+    pooled = np.zeros((B, Hq, n), dtype=np.float64)
+
+    wanted = None if heads is None else set(heads)
+
+    def unit(bc):
+        b, c = bc
+        hs = [h for h in range(c * g, (c + 1) * g) if wanted is None or (b, h) in wanted]
+        if not hs:
+            return
+        kf = bf16_bits_to_f64(k[b, c])
+        for h in hs:
+            vt = window_votes(bf16_bits_to_f64(q_obs[b, h]), kf)
+            pv = pool1d(vt, pool_kernel, pool_type)
+            idx = topk_positions(pv, ksel)
+            vote[b, h] = vt
+            pooled[b, h] = pv
+            out_idx[b, h] = idx
+            out_k[b, h, :ksel] = k[b, c, idx]
+            out_v[b, h, :ksel] = v[b, c, idx]
+            out_k[b, h, ksel:] = k[b, c, n:]
+            out_v[b, h, ksel:] = v[b, c, n:]
+
+    units = [(b, c) for b in range(B) for c in range(Hkv)]
+    if workers > 1:
+        with ThreadPoolExecutor(max_workers=workers) as ex:
+            list(ex.map(unit, units))
+    else:
+        for u in units:
+            unit(u)
+    return {"out_k": out_k, "out_v": out_v, "out_idx": out_idx, "vote": vote, "pooled": pooled}
