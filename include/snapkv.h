@@ -1,0 +1,158 @@
+/*
+ * snapkv.h - C ABI of the SnapKV prompt KV-cache compression step for NVIDIA B200.
+ *
+ * The step follows arXiv 2404.14469, Sec. 4 (Eq. 1-2) and Listing 1: the last W
+ * prompt queries (the observation window) score every prompt key, the softmax
+ * probabilities are summed over the window, pooled along the sequence, the
+ * top-(budget - W) prefix positions are chosen per head, and those K/V rows plus
+ * the window's own rows form the compressed cache.
+ *
+ * Notation: L prompt length, W window, n = L - W prefix length, d head dimension,
+ * ksel = budget - W selected rows per head, g = Hq / Hkv (query head h reads KV
+ * head h / g; each query head selects its own positions).
+ *
+ * Conventions for every entry point
+ *   - All tensors are dense, row-major, in the stated shape; "bf16" is the 16-bit
+ *     brain-float bit pattern.  Device pointers must be 16-byte aligned and must
+ *     not alias one another.
+ *   - The caller owns every buffer.  The library allocates no device memory and
+ *     keeps no per-call state; it only caches, per process, driver entry points.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     default stream).  Calls return without synchronising unless stated.
+ *   - Errors come back as a snapkv_status_t; nothing aborts or throws.  Argument
+ *     errors are found on the host before anything is launched.
+ *   - A device-side wait that exceeds its time limit stops the kernel early and
+ *     records SNAPKV_ERR_TIMEOUT in the first word of the workspace; read it with
+ *     snapkv_device_status after the stream has drained.
+ */
+#ifndef SNAPKV_H_
+#define SNAPKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SNAPKV_OK = 0,
+  SNAPKV_ERR_INVALID_ARG = 1, /* a size, enum or pointer is not acceptable            */
+  SNAPKV_ERR_UNSUPPORTED = 2, /* valid for the method, not implemented by the kernels  */
+  SNAPKV_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small            */
+  SNAPKV_ERR_CUDA = 4,        /* a CUDA runtime/driver call or a launch failed         */
+  SNAPKV_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up                    */
+} snapkv_status_t;
+
+enum { SNAPKV_POOL_MAX = 0, SNAPKV_POOL_AVG = 1 };
+
+/* Supported range: d in {64, 128}; 1 <= W <= 128 and W <= L; pool_kernel odd in
+ * [1, 63]; W < budget; Hq % Hkv == 0; B*Hkv*L*d < 2^40.  Anything else that is
+ * meaningful for the method returns SNAPKV_ERR_UNSUPPORTED, anything meaningless
+ * SNAPKV_ERR_INVALID_ARG. */
+
+/* Human-readable name of a status code (static storage). */
+const char* snapkv_status_string(int status);
+
+/* Rows written per head by snapkv_compress: min(budget, L).  Listing 1 returns the
+ * cache unchanged when the prompt is not longer than the budget.  Host only. */
+int snapkv_out_rows(int L, int budget);
+
+/* Bytes of device scratch snapkv_compress / snapkv_window_scores / snapkv_pool_topk
+ * need for these sizes (the maximum over the three); 0 if the arguments are not
+ * acceptable.  Host only, no CUDA calls.  The workspace must be 256-byte aligned. */
+size_t snapkv_workspace_size(int B, int Hq, int Hkv, int L, int d, int W,
+                             int pool_kernel, int pool_type, int budget);
+
+/*
+ * The whole step (Listing 1; Sec. 4.1 "vote" then "update and store").
+ *   q_obs   bf16 [B, Hq, W, d]   device  the last W prompt queries (post-RoPE)
+ *   k, v    bf16 [B, Hkv, L, d]  device  prompt keys / values as cached
+ *   out_k/v bf16 [B, Hq, budget, d] device.  Per head: rows [0, ksel) are the selected
+ *           prefix rows in ascending position, rows [ksel, budget) the window rows.
+ *   out_idx int32 [B, Hq, budget - W] device: the selected prefix positions,
+ *           strictly ascending, each in [0, n).
+ * Logits are q.k/sqrt(d) with a causal mask inside the window; the softmax
+ * normaliser covers every visible key; average pooling divides by pool_kernel;
+ * ties go to the lower position.
+ * If budget >= L the cache is copied through (expanded to Hq heads): per head rows
+ * [0, L) of out_k/out_v are written with row stride unchanged (budget rows per
+ * head), out_idx[..., 0:n] = 0..n-1 (row stride budget - W), everything else is
+ * left untouched.
+ */
+snapkv_status_t snapkv_compress(const void* q_obs, const void* k, const void* v,
+                                int B, int Hq, int Hkv, int L, int d, int W,
+                                int pool_kernel, int pool_type, int budget,
+                                void* out_k, void* out_v, int32_t* out_idx,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Steps "score" and "vote" alone (Eq. 1; Listing 1's compute_attn and .sum):
+ *   out_vote fp32 [B, Hq, n] device, vote[j] = sum over window rows i of
+ *   softmax_i(q_i.k/sqrt(d))[j], j in [0, n).  fp32 accumulation of bf16 products.
+ * Requires W < L.
+ */
+snapkv_status_t snapkv_window_scores(const void* q_obs, const void* k,
+                                     int B, int Hq, int Hkv, int L, int d, int W,
+                                     float* out_vote,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Steps "pool" and "top-k" alone (Listing 1's pool1d and topk; Eq. 2) on `rows`
+ * independent rows:
+ *   vote    fp32 [rows, n] device, finite and >= 0
+ *   out_idx int32 [rows, ksel] device, ascending positions of the ksel largest pooled
+ *           votes; among equal pooled votes the lower positions win.
+ * Requires 1 <= ksel <= n.  `workspace` must hold snapkv_pool_topk_workspace_size
+ * bytes (may be NULL when that is 0).
+ */
+size_t snapkv_pool_topk_workspace_size(int rows, int n);
+snapkv_status_t snapkv_pool_topk(const float* vote, int rows, int n,
+                                 int pool_kernel, int pool_type, int ksel,
+                                 int32_t* out_idx,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Step "gather + append" alone (Listing 1's gather and cat): with idx int32
+ * [B, Hq, ksel] device (positions in [0, L - W)), writes per head the rows k[idx],
+ * then the last W rows of k, to out_k [B, Hq, ksel + W, d]; same for v.
+ * Byte copies: bit-exact.
+ */
+snapkv_status_t snapkv_gather(const void* k, const void* v, const int32_t* idx,
+                              int B, int Hq, int Hkv, int L, int d, int W, int ksel,
+                              void* out_k, void* out_v, void* stream);
+
+/*
+ * snapkv_compress for callers whose tensors live in host memory (pinned memory
+ * gives asynchronous copies).  q_obs, k, v, out_k, out_v, out_idx are HOST pointers
+ * with the shapes above (out_k/out_v [B,Hq,budget,d], out_idx [B,Hq,budget-W]).
+ * `staging` is DEVICE scratch of at least snapkv_host_staging_size(...) bytes,
+ * 256-byte aligned, holding the device copies and the workspace.  Copies in,
+ * compresses, copies out, all on `stream`; returns after enqueueing (synchronise
+ * the stream before reading the outputs).
+ */
+size_t snapkv_host_staging_size(int B, int Hq, int Hkv, int L, int d, int W,
+                                int pool_kernel, int pool_type, int budget);
+snapkv_status_t snapkv_compress_host(const void* q_obs, const void* k, const void* v,
+                                     int B, int Hq, int Hkv, int L, int d, int W,
+                                     int pool_kernel, int pool_type, int budget,
+                                     void* out_k, void* out_v, int32_t* out_idx,
+                                     void* staging, size_t staging_bytes, void* stream);
+
+/*
+ * Synchronises `stream`, reads the status word the kernels keep at the start of
+ * `workspace` and returns it (SNAPKV_OK or SNAPKV_ERR_TIMEOUT), or SNAPKV_ERR_CUDA
+ * if the stream reports an error.  `detail`, if not NULL, receives a code telling
+ * which wait gave up (0 if none).
+ */
+snapkv_status_t snapkv_device_status(const void* workspace, void* stream, int* detail);
+
+/* Number of kernel launches the last successful snapkv_compress /
+ * snapkv_window_scores call of this thread enqueued (for accounting in benchmarks).
+ * Host only. */
+int snapkv_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SNAPKV_H_ */

@@ -1,0 +1,70 @@
+// Internal interfaces between the translation units of libsnapkv (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace snapkv {
+
+constexpr int TILE_KEYS = 128;      // keys per MMA tile
+constexpr int MAX_COLS = 128;       // window-query columns handled by one unit
+constexpr int STATUS_BYTES = 256;   // status block at the start of every workspace
+constexpr int SM_COUNT_HINT = 148;  // B200
+
+// Codes stored in the workspace status block's second word when a wait gives up.
+enum WaitCode {
+  WAIT_NONE = 0,
+  WAIT_PRODUCER_EMPTY = 1,
+  WAIT_MMA_FULL = 2,
+  WAIT_MMA_TMEM_EMPTY = 3,
+  WAIT_EPI_TMEM_FULL = 4,
+  WAIT_Q_FULL = 5,
+  WAIT_DRAIN = 6,
+};
+
+// How the scoring passes split the work.  A "unit" is one (batch, KV head, head
+// sub-group): `hpu` query heads that share the KV head, hpu * W <= MAX_COLS columns.
+struct ScorePlan {
+  int g;            // Hq / Hkv
+  int hpu;          // query heads per unit
+  int sub_per_kv;   // g / hpu
+  int units;        // B * Hkv * sub_per_kv
+  int ncols;        // hpu * W
+  int npad;         // ncols rounded up to 32, 64 or 128
+  int tiles_stats;  // ceil(L / TILE_KEYS): the normaliser covers every key
+  int tiles_vote;   // ceil(n / TILE_KEYS): votes exist for prefix keys only
+  int units_per_wave;
+  int chunks_stats; // CTAs per unit in the statistics pass
+  int chunks_vote;  // CTAs per unit in the vote pass
+};
+
+struct WorkspaceLayout {
+  size_t off_status, off_counters, off_partials, off_lse, off_vote, off_pooled, total;
+};
+
+bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* plan);
+WorkspaceLayout make_layout(const ScorePlan& p, int B, int Hq, int n, bool need_vote,
+                            bool need_pooled);
+bool select_needs_scratch(int n);
+
+// Enqueue both scoring passes.  `vote` is fp32 [B*Hq, n].
+cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv, int L,
+                                 int d, int W, const ScorePlan& plan, float* vote, int* status,
+                                 int* counters, float2* partials, float* lse2, cudaStream_t stream,
+                                 int* launches);
+
+// Pool + top-k over `rows` rows of fp32 votes.  `pooled_scratch` (fp32 [rows, n]) is
+// only touched when select_needs_scratch(n).
+cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel, int pool_type,
+                             int ksel, int32_t* out_idx, float* pooled_scratch,
+                             cudaStream_t stream, int* launches);
+
+// Gather + append.  idx == nullptr copies rows 0..ksel-1 (identity path).
+cudaError_t launch_gather(const void* k, const void* v, const int32_t* idx, int B, int Hq, int Hkv,
+                          int L, int d, int W, int ksel, int out_rows_stride, void* out_k,
+                          void* out_v, cudaStream_t stream, int* launches);
+
+cudaError_t launch_iota_idx(int32_t* out_idx, int rows, int n, int row_stride, cudaStream_t stream,
+                            int* launches);
+
+}  // namespace snapkv
