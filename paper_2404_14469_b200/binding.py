@@ -1,0 +1,226 @@
+"""ctypes binding of libsnapkv.so: argument marshalling only.
+
+Every step of the compression path runs in the library's CUDA kernels; torch is
+used here for device memory (outputs, workspace) and for the current stream.  The
+functions carry the names of the C entry points declared in include/snapkv.h.
+If the library has not been built, or a call returns an error status, a
+RuntimeError is raised: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libsnapkv.so")
+
+POOL_MAX = 0
+POOL_AVG = 1
+OK = 0
+
+SYMBOLS = [
+    "snapkv_status_string", "snapkv_out_rows", "snapkv_workspace_size", "snapkv_compress",
+    "snapkv_window_scores", "snapkv_pool_topk_workspace_size", "snapkv_pool_topk", "snapkv_gather",
+    "snapkv_host_staging_size", "snapkv_compress_host", "snapkv_device_status",
+    "snapkv_last_launch_count",
+]
+
+_lib = None
+
+
+class SnapKVError(RuntimeError):
+    pass
+
+
+def lib() -> ctypes.CDLL:
+    """Load the shared library (once); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise SnapKVError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2404_14469_b200.build` "
+            "(there is no CPU or framework fallback)")
+    L = ctypes.CDLL(LIB_PATH)
+    c_int, c_sz, c_vp = ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p
+    L.snapkv_status_string.restype = ctypes.c_char_p
+    L.snapkv_status_string.argtypes = [c_int]
+    L.snapkv_out_rows.restype = c_int
+    L.snapkv_out_rows.argtypes = [c_int, c_int]
+    L.snapkv_workspace_size.restype = c_sz
+    L.snapkv_workspace_size.argtypes = [c_int] * 9
+    L.snapkv_compress.restype = c_int
+    L.snapkv_compress.argtypes = [c_vp] * 3 + [c_int] * 9 + [c_vp] * 3 + [c_vp, c_sz, c_vp]
+    L.snapkv_window_scores.restype = c_int
+    L.snapkv_window_scores.argtypes = [c_vp] * 2 + [c_int] * 6 + [c_vp, c_vp, c_sz, c_vp]
+    L.snapkv_pool_topk_workspace_size.restype = c_sz
+    L.snapkv_pool_topk_workspace_size.argtypes = [c_int, c_int]
+    L.snapkv_pool_topk.restype = c_int
+    L.snapkv_pool_topk.argtypes = [c_vp] + [c_int] * 5 + [c_vp, c_vp, c_sz, c_vp]
+    L.snapkv_gather.restype = c_int
+    L.snapkv_gather.argtypes = [c_vp] * 3 + [c_int] * 7 + [c_vp] * 3
+    L.snapkv_host_staging_size.restype = c_sz
+    L.snapkv_host_staging_size.argtypes = [c_int] * 9
+    L.snapkv_compress_host.restype = c_int
+    L.snapkv_compress_host.argtypes = [c_vp] * 3 + [c_int] * 9 + [c_vp] * 3 + [c_vp, c_sz, c_vp]
+    L.snapkv_device_status.restype = c_int
+    L.snapkv_device_status.argtypes = [c_vp, c_vp, ctypes.POINTER(c_int)]
+    L.snapkv_last_launch_count.restype = c_int
+    L.snapkv_last_launch_count.argtypes = []
+    _lib = L
+    return L
+
+
+def status_string(code: int) -> str:
+    return lib().snapkv_status_string(int(code)).decode()
+
+
+def _check(code: int, what: str):
+    if code != OK:
+        raise SnapKVError(f"{what} failed: {status_string(code)}")
+
+
+def _stream_ptr() -> int:
+    return int(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev_bf16(t: torch.Tensor, name: str) -> torch.Tensor:
+    if not (t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()):
+        raise SnapKVError(f"{name} must be a contiguous CUDA bf16 tensor")
+    return t
+
+
+def _shapes(q_obs, k):
+    B, Hq, W, d = q_obs.shape
+    Bk, Hkv, L, dk = k.shape
+    if Bk != B or dk != d:
+        raise SnapKVError("q_obs and k disagree on batch or head dimension")
+    return B, Hq, Hkv, L, d, W
+
+
+def _alloc_ws(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def snapkv_out_rows(L: int, budget: int) -> int:
+    return lib().snapkv_out_rows(L, budget)
+
+
+def snapkv_workspace_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget) -> int:
+    return lib().snapkv_workspace_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget)
+
+
+def snapkv_compress(q_obs, k, v, pool_kernel: int, pool_type: int, budget: int,
+                    out_k=None, out_v=None, out_idx=None, workspace=None):
+    """Whole step on device tensors.  Returns (out_k, out_v, out_idx, workspace).
+
+    out_k/out_v: bf16 [B, Hq, min(budget, L), d]; out_idx: int32 [B, Hq, rows - W].
+    """
+    _dev_bf16(q_obs, "q_obs"), _dev_bf16(k, "k"), _dev_bf16(v, "v")
+    B, Hq, Hkv, L, d, W = _shapes(q_obs, k)
+    L_ = lib()
+    rows = L_.snapkv_out_rows(L, budget)
+    # the library addresses outputs with `budget` rows per head; on the identity path we
+    # call it with budget = L so that the tensors stay dense
+    eff_budget = rows
+    dev = k.device
+    if out_k is None:
+        out_k = torch.empty(B, Hq, rows, d, dtype=torch.bfloat16, device=dev)
+    if out_v is None:
+        out_v = torch.empty(B, Hq, rows, d, dtype=torch.bfloat16, device=dev)
+    if out_idx is None:
+        out_idx = torch.empty(B, Hq, rows - W, dtype=torch.int32, device=dev)
+    need = L_.snapkv_workspace_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, eff_budget)
+    if workspace is None or workspace.numel() < need:
+        workspace = _alloc_ws(need, dev)
+    code = L_.snapkv_compress(q_obs.data_ptr(), k.data_ptr(), v.data_ptr(), B, Hq, Hkv, L, d, W,
+                              pool_kernel, pool_type, eff_budget, out_k.data_ptr(), out_v.data_ptr(),
+                              out_idx.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                              _stream_ptr())
+    _check(code, "snapkv_compress")
+    return out_k, out_v, out_idx, workspace
+
+
+def snapkv_window_scores(q_obs, k, out_vote=None, workspace=None):
+    """Votes fp32 [B, Hq, n].  Returns (out_vote, workspace)."""
+    _dev_bf16(q_obs, "q_obs"), _dev_bf16(k, "k")
+    B, Hq, Hkv, L, d, W = _shapes(q_obs, k)
+    L_ = lib()
+    dev = k.device
+    if out_vote is None:
+        out_vote = torch.empty(B, Hq, L - W, dtype=torch.float32, device=dev)
+    need = L_.snapkv_workspace_size(B, Hq, Hkv, L, d, W, 1, 0, W + 1)
+    if workspace is None or workspace.numel() < need:
+        workspace = _alloc_ws(need, dev)
+    code = L_.snapkv_window_scores(q_obs.data_ptr(), k.data_ptr(), B, Hq, Hkv, L, d, W,
+                                   out_vote.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                   _stream_ptr())
+    _check(code, "snapkv_window_scores")
+    return out_vote, workspace
+
+
+def snapkv_pool_topk(vote, pool_kernel: int, pool_type: int, ksel: int, out_idx=None,
+                     workspace=None):
+    """vote fp32 [rows, n] (CUDA) -> int32 [rows, ksel] ascending positions."""
+    if not (vote.is_cuda and vote.dtype == torch.float32 and vote.is_contiguous() and vote.dim() == 2):
+        raise SnapKVError("vote must be a contiguous CUDA fp32 [rows, n] tensor")
+    rows, n = vote.shape
+    L_ = lib()
+    if out_idx is None:
+        out_idx = torch.empty(rows, max(ksel, 0), dtype=torch.int32, device=vote.device)
+    need = L_.snapkv_pool_topk_workspace_size(rows, n)
+    if need and (workspace is None or workspace.numel() < need):
+        workspace = _alloc_ws(need, vote.device)
+    code = L_.snapkv_pool_topk(vote.data_ptr(), rows, n, pool_kernel, pool_type, ksel,
+                               out_idx.data_ptr(), workspace.data_ptr() if workspace is not None else None,
+                               workspace.numel() if workspace is not None else 0, _stream_ptr())
+    _check(code, "snapkv_pool_topk")
+    return out_idx
+
+
+def snapkv_gather(k, v, idx, W: int):
+    """k, v bf16 [B,Hkv,L,d]; idx int32 [B,Hq,ksel] -> out_k, out_v [B,Hq,ksel+W,d]."""
+    _dev_bf16(k, "k"), _dev_bf16(v, "v")
+    if not (idx.is_cuda and idx.dtype == torch.int32 and idx.is_contiguous()):
+        raise SnapKVError("idx must be a contiguous CUDA int32 tensor")
+    B, Hkv, L, d = k.shape
+    _, Hq, ksel = idx.shape
+    out_k = torch.empty(B, Hq, ksel + W, d, dtype=torch.bfloat16, device=k.device)
+    out_v = torch.empty_like(out_k)
+    code = lib().snapkv_gather(k.data_ptr(), v.data_ptr(), idx.data_ptr(), B, Hq, Hkv, L, d, W, ksel,
+                               out_k.data_ptr(), out_v.data_ptr(), _stream_ptr())
+    _check(code, "snapkv_gather")
+    return out_k, out_v
+
+
+def snapkv_host_staging_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget) -> int:
+    return lib().snapkv_host_staging_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget)
+
+
+def snapkv_compress_host(q_obs, k, v, pool_kernel, pool_type, budget, out_k, out_v, out_idx,
+                         staging):
+    """Host (ideally pinned) tensors in and out; `staging` is a CUDA uint8 tensor.
+    Enqueues copies and kernels on the current stream and returns without synchronising."""
+    for t, name in ((q_obs, "q_obs"), (k, "k"), (v, "v"), (out_k, "out_k"), (out_v, "out_v"),
+                    (out_idx, "out_idx")):
+        if t.is_cuda or not t.is_contiguous():
+            raise SnapKVError(f"{name} must be a contiguous host tensor")
+    B, Hq, Hkv, L, d, W = _shapes(q_obs, k)
+    code = lib().snapkv_compress_host(q_obs.data_ptr(), k.data_ptr(), v.data_ptr(), B, Hq, Hkv, L, d,
+                                      W, pool_kernel, pool_type, budget, out_k.data_ptr(),
+                                      out_v.data_ptr(), out_idx.data_ptr(), staging.data_ptr(),
+                                      staging.numel(), _stream_ptr())
+    _check(code, "snapkv_compress_host")
+
+
+def snapkv_device_status(workspace):
+    """Synchronises the current stream; returns (status, detail)."""
+    detail = ctypes.c_int(0)
+    code = lib().snapkv_device_status(workspace.data_ptr(), _stream_ptr(), ctypes.byref(detail))
+    return code, detail.value
+
+
+def snapkv_last_launch_count() -> int:
+    return lib().snapkv_last_launch_count()

@@ -1,0 +1,273 @@
+// C ABI of libsnapkv: argument validation, workspace layout, and the sequence of
+// launches that makes up the compression step (Listing 1).
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/snapkv.h"
+#include "snapkv_internal.h"
+
+namespace snapkv {
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+WorkspaceLayout make_layout(const ScorePlan& p, int B, int Hq, int n, bool need_vote,
+                            bool need_pooled) {
+  WorkspaceLayout w;
+  size_t off = 0;
+  w.off_status = off;
+  off += STATUS_BYTES;
+  w.off_counters = off;
+  off = align_up(off + sizeof(int) * static_cast<size_t>(p.units), 256);
+  w.off_partials = off;
+  off = align_up(off + sizeof(float2) * static_cast<size_t>(p.units) * p.chunks_stats * MAX_COLS, 256);
+  w.off_lse = off;
+  off = align_up(off + sizeof(float) * static_cast<size_t>(p.units) * MAX_COLS, 256);
+  w.off_vote = off;
+  const size_t row_bytes = sizeof(float) * static_cast<size_t>(B) * Hq * (n > 0 ? n : 0);
+  if (need_vote) off = align_up(off + row_bytes, 256);
+  w.off_pooled = off;
+  if (need_pooled) off = align_up(off + row_bytes, 256);
+  w.total = off;
+  return w;
+}
+
+static thread_local int g_last_launches = 0;
+
+static snapkv_status_t check_common(int B, int Hq, int Hkv, int L, int d, int W) {
+  if (B < 1 || Hq < 1 || Hkv < 1 || L < 1 || d < 1 || W < 1) return SNAPKV_ERR_INVALID_ARG;
+  if (Hq % Hkv != 0 || W > L) return SNAPKV_ERR_INVALID_ARG;
+  if (d != 64 && d != 128) return SNAPKV_ERR_UNSUPPORTED;
+  if (W > MAX_COLS) return SNAPKV_ERR_UNSUPPORTED;
+  if (static_cast<double>(B) * Hkv * L * d >= 1099511627776.0) return SNAPKV_ERR_UNSUPPORTED;
+  if (static_cast<double>(B) * Hq * L >= 2147483647.0 * 16) return SNAPKV_ERR_UNSUPPORTED;
+  return SNAPKV_OK;
+}
+
+static snapkv_status_t check_pool(int pool_kernel, int pool_type) {
+  if (pool_kernel < 1 || (pool_kernel & 1) == 0) return SNAPKV_ERR_INVALID_ARG;
+  if (pool_type != SNAPKV_POOL_MAX && pool_type != SNAPKV_POOL_AVG) return SNAPKV_ERR_INVALID_ARG;
+  if (pool_kernel > 63) return SNAPKV_ERR_UNSUPPORTED;
+  return SNAPKV_OK;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace snapkv
+
+using namespace snapkv;
+
+extern "C" {
+
+const char* snapkv_status_string(int status) {
+  switch (status) {
+    case SNAPKV_OK: return "SNAPKV_OK";
+    case SNAPKV_ERR_INVALID_ARG: return "SNAPKV_ERR_INVALID_ARG";
+    case SNAPKV_ERR_UNSUPPORTED: return "SNAPKV_ERR_UNSUPPORTED";
+    case SNAPKV_ERR_WORKSPACE: return "SNAPKV_ERR_WORKSPACE";
+    case SNAPKV_ERR_CUDA: return "SNAPKV_ERR_CUDA";
+    case SNAPKV_ERR_TIMEOUT: return "SNAPKV_ERR_TIMEOUT";
+    default: return "SNAPKV_UNKNOWN_STATUS";
+  }
+}
+
+int snapkv_out_rows(int L, int budget) { return budget < L ? budget : L; }
+
+int snapkv_last_launch_count(void) { return g_last_launches; }
+
+size_t snapkv_workspace_size(int B, int Hq, int Hkv, int L, int d, int W, int pool_kernel,
+                             int pool_type, int budget) {
+  if (check_common(B, Hq, Hkv, L, d, W) != SNAPKV_OK) return 0;
+  if (check_pool(pool_kernel, pool_type) != SNAPKV_OK) return 0;
+  if (budget <= W) return 0;
+  ScorePlan p;
+  if (!make_score_plan(B, Hq, Hkv, L, d, W, &p)) return 0;
+  const int n = L - W;
+  return make_layout(p, B, Hq, n, true, select_needs_scratch(n)).total;
+}
+
+size_t snapkv_pool_topk_workspace_size(int rows, int n) {
+  if (rows < 1 || n < 1) return 0;
+  return select_needs_scratch(n) ? sizeof(float) * static_cast<size_t>(rows) * n : 0;
+}
+
+snapkv_status_t snapkv_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv,
+                                     int L, int d, int W, float* out_vote, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+  snapkv_status_t st = check_common(B, Hq, Hkv, L, d, W);
+  if (st != SNAPKV_OK) return st;
+  if (W >= L) return SNAPKV_ERR_INVALID_ARG;
+  if (!q_obs || !k || !out_vote) return SNAPKV_ERR_INVALID_ARG;
+  if (!aligned16(q_obs) || !aligned16(k) || (reinterpret_cast<uintptr_t>(out_vote) & 3))
+    return SNAPKV_ERR_INVALID_ARG;
+  ScorePlan p;
+  if (!make_score_plan(B, Hq, Hkv, L, d, W, &p)) return SNAPKV_ERR_UNSUPPORTED;
+  const WorkspaceLayout w = make_layout(p, B, Hq, L - W, false, false);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < w.total)
+    return SNAPKV_ERR_WORKSPACE;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(ws + w.off_status, 0, STATUS_BYTES, s) != cudaSuccess) return SNAPKV_ERR_CUDA;
+  int launches = 0;
+  cudaError_t e = launch_window_scores(
+      q_obs, k, B, Hq, Hkv, L, d, W, p, out_vote, reinterpret_cast<int*>(ws + w.off_status),
+      reinterpret_cast<int*>(ws + w.off_counters), reinterpret_cast<float2*>(ws + w.off_partials),
+      reinterpret_cast<float*>(ws + w.off_lse), s, &launches);
+  if (e != cudaSuccess) return SNAPKV_ERR_CUDA;
+  g_last_launches = launches;
+  return SNAPKV_OK;
+}
+
+snapkv_status_t snapkv_pool_topk(const float* vote, int rows, int n, int pool_kernel, int pool_type,
+                                 int ksel, int32_t* out_idx, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
+  if (rows < 1 || n < 1 || ksel < 1 || ksel > n || !vote || !out_idx) return SNAPKV_ERR_INVALID_ARG;
+  snapkv_status_t st = check_pool(pool_kernel, pool_type);
+  if (st != SNAPKV_OK) return st;
+  const size_t need = snapkv_pool_topk_workspace_size(rows, n);
+  if (need > 0 &&
+      (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < need))
+    return SNAPKV_ERR_WORKSPACE;
+  int launches = 0;
+  cudaError_t e = launch_pool_topk(vote, rows, n, pool_kernel, pool_type, ksel, out_idx,
+                                   static_cast<float*>(workspace),
+                                   static_cast<cudaStream_t>(stream), &launches);
+  return e == cudaSuccess ? SNAPKV_OK : SNAPKV_ERR_CUDA;
+}
+
+snapkv_status_t snapkv_gather(const void* k, const void* v, const int32_t* idx, int B, int Hq,
+                              int Hkv, int L, int d, int W, int ksel, void* out_k, void* out_v,
+                              void* stream) {
+  snapkv_status_t st = check_common(B, Hq, Hkv, L, d, W);
+  if (st != SNAPKV_OK) return st;
+  if (ksel < 0 || ksel > L - W || !k || !v || !out_k || !out_v || (ksel > 0 && !idx))
+    return SNAPKV_ERR_INVALID_ARG;
+  if (!aligned16(k) || !aligned16(v) || !aligned16(out_k) || !aligned16(out_v))
+    return SNAPKV_ERR_INVALID_ARG;
+  int launches = 0;
+  cudaError_t e = launch_gather(k, v, idx, B, Hq, Hkv, L, d, W, ksel, ksel + W, out_k, out_v,
+                                static_cast<cudaStream_t>(stream), &launches);
+  return e == cudaSuccess ? SNAPKV_OK : SNAPKV_ERR_CUDA;
+}
+
+snapkv_status_t snapkv_compress(const void* q_obs, const void* k, const void* v, int B, int Hq,
+                                int Hkv, int L, int d, int W, int pool_kernel, int pool_type,
+                                int budget, void* out_k, void* out_v, int32_t* out_idx,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  snapkv_status_t st = check_common(B, Hq, Hkv, L, d, W);
+  if (st != SNAPKV_OK) return st;
+  st = check_pool(pool_kernel, pool_type);
+  if (st != SNAPKV_OK) return st;
+  if (budget <= W) return SNAPKV_ERR_INVALID_ARG;
+  if (!q_obs || !k || !v || !out_k || !out_v) return SNAPKV_ERR_INVALID_ARG;
+  if (!aligned16(q_obs) || !aligned16(k) || !aligned16(v) || !aligned16(out_k) || !aligned16(out_v))
+    return SNAPKV_ERR_INVALID_ARG;
+  const int n = L - W;
+  if (!out_idx && n > 0) return SNAPKV_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int launches = 0;
+  if (budget >= L) {
+    // Listing 1's early return: nothing is dropped, the cache is expanded to Hq heads.
+    if (launch_iota_idx(out_idx, B * Hq, n, budget - W, s, &launches) != cudaSuccess)
+      return SNAPKV_ERR_CUDA;
+    if (launch_gather(k, v, nullptr, B, Hq, Hkv, L, d, W, n, budget, out_k, out_v, s, &launches) !=
+        cudaSuccess)
+      return SNAPKV_ERR_CUDA;
+    g_last_launches = launches;
+    return SNAPKV_OK;
+  }
+  ScorePlan p;
+  if (!make_score_plan(B, Hq, Hkv, L, d, W, &p)) return SNAPKV_ERR_UNSUPPORTED;
+  const bool scratch = select_needs_scratch(n);
+  const WorkspaceLayout w = make_layout(p, B, Hq, n, true, scratch);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < w.total)
+    return SNAPKV_ERR_WORKSPACE;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  if (cudaMemsetAsync(ws + w.off_status, 0, STATUS_BYTES, s) != cudaSuccess) return SNAPKV_ERR_CUDA;
+  float* vote = reinterpret_cast<float*>(ws + w.off_vote);
+  const int ksel = budget - W;
+  if (launch_window_scores(q_obs, k, B, Hq, Hkv, L, d, W, p, vote,
+                           reinterpret_cast<int*>(ws + w.off_status),
+                           reinterpret_cast<int*>(ws + w.off_counters),
+                           reinterpret_cast<float2*>(ws + w.off_partials),
+                           reinterpret_cast<float*>(ws + w.off_lse), s, &launches) != cudaSuccess)
+    return SNAPKV_ERR_CUDA;
+  if (launch_pool_topk(vote, B * Hq, n, pool_kernel, pool_type, ksel, out_idx,
+                       scratch ? reinterpret_cast<float*>(ws + w.off_pooled) : nullptr, s,
+                       &launches) != cudaSuccess)
+    return SNAPKV_ERR_CUDA;
+  if (launch_gather(k, v, out_idx, B, Hq, Hkv, L, d, W, ksel, budget, out_k, out_v, s, &launches) !=
+      cudaSuccess)
+    return SNAPKV_ERR_CUDA;
+  g_last_launches = launches;
+  return SNAPKV_OK;
+}
+
+size_t snapkv_host_staging_size(int B, int Hq, int Hkv, int L, int d, int W, int pool_kernel,
+                                int pool_type, int budget) {
+  if (check_common(B, Hq, Hkv, L, d, W) != SNAPKV_OK) return 0;
+  if (check_pool(pool_kernel, pool_type) != SNAPKV_OK || budget <= W) return 0;
+  const size_t qb = align_up(static_cast<size_t>(B) * Hq * W * d * 2, 256);
+  const size_t kb = align_up(static_cast<size_t>(B) * Hkv * L * d * 2, 256);
+  const size_t ob = align_up(static_cast<size_t>(B) * Hq * budget * d * 2, 256);
+  const size_t ib = align_up(static_cast<size_t>(B) * Hq * (budget - W) * 4, 256);
+  size_t ws = 0;
+  if (budget < L) ws = snapkv_workspace_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget);
+  return qb + 2 * kb + 2 * ob + ib + align_up(ws, 256);
+}
+
+snapkv_status_t snapkv_compress_host(const void* q_obs, const void* k, const void* v, int B, int Hq,
+                                     int Hkv, int L, int d, int W, int pool_kernel, int pool_type,
+                                     int budget, void* out_k, void* out_v, int32_t* out_idx,
+                                     void* staging, size_t staging_bytes, void* stream) {
+  const size_t need =
+      snapkv_host_staging_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget);
+  if (need == 0) {
+    snapkv_status_t st = check_common(B, Hq, Hkv, L, d, W);
+    if (st != SNAPKV_OK) return st;
+    st = check_pool(pool_kernel, pool_type);
+    return st != SNAPKV_OK ? st : SNAPKV_ERR_INVALID_ARG;
+  }
+  if (!q_obs || !k || !v || !out_k || !out_v || !out_idx) return SNAPKV_ERR_INVALID_ARG;
+  if (!staging || (reinterpret_cast<uintptr_t>(staging) & 255) || staging_bytes < need)
+    return SNAPKV_ERR_WORKSPACE;
+  const size_t q_raw = static_cast<size_t>(B) * Hq * W * d * 2;
+  const size_t k_raw = static_cast<size_t>(B) * Hkv * L * d * 2;
+  const size_t o_raw = static_cast<size_t>(B) * Hq * budget * d * 2;
+  const size_t i_raw = static_cast<size_t>(B) * Hq * (budget - W) * 4;
+  uint8_t* p = static_cast<uint8_t*>(staging);
+  uint8_t* dq = p; p += align_up(q_raw, 256);
+  uint8_t* dk = p; p += align_up(k_raw, 256);
+  uint8_t* dv = p; p += align_up(k_raw, 256);
+  uint8_t* dok = p; p += align_up(o_raw, 256);
+  uint8_t* dov = p; p += align_up(o_raw, 256);
+  uint8_t* di = p; p += align_up(i_raw, 256);
+  uint8_t* dws = p;
+  const size_t ws_bytes = staging_bytes - static_cast<size_t>(dws - static_cast<uint8_t*>(staging));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(dq, q_obs, q_raw, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(dk, k, k_raw, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(dv, v, k_raw, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return SNAPKV_ERR_CUDA;
+  snapkv_status_t st =
+      snapkv_compress(dq, dk, dv, B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget, dok, dov,
+                      reinterpret_cast<int32_t*>(di), dws, ws_bytes, stream);
+  if (st != SNAPKV_OK) return st;
+  if (cudaMemcpyAsync(out_k, dok, o_raw, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaMemcpyAsync(out_v, dov, o_raw, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaMemcpyAsync(out_idx, di, i_raw, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return SNAPKV_ERR_CUDA;
+  return SNAPKV_OK;
+}
+
+snapkv_status_t snapkv_device_status(const void* workspace, void* stream, int* detail) {
+  if (!workspace) return SNAPKV_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int host[2] = {0, 0};
+  if (cudaMemcpyAsync(host, workspace, sizeof(host), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return SNAPKV_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return SNAPKV_ERR_CUDA;
+  if (detail) *detail = host[1];
+  return host[0] == 0 ? SNAPKV_OK : static_cast<snapkv_status_t>(host[0]);
+}
+
+}  // extern "C"

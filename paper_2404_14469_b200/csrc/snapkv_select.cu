@@ -1,0 +1,217 @@
+// Pooling and per-head top-k (Listing 1's pool1d and topk; Eq. 2), one CTA per row.
+//
+//  1. pooled[j] = max or mean of vote[j-r .. j+r] (stride 1, same length; the mean
+//     divides by pool_kernel, positions outside the row count as zero), turned into a
+//     32-bit key whose unsigned order is the float order.  Keys stay in shared memory
+//     when the row fits, otherwise in caller-provided global scratch.
+//  2. radix select of the ksel-th largest key: three histogram passes (11 + 11 + 10
+//     bits), each followed by a block scan from the top bin down.
+//  3. ordered compaction: every key above the threshold, plus the lowest-position keys
+//     equal to it until ksel are taken, written in ascending position.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "snapkv_internal.h"
+
+namespace snapkv {
+
+namespace {
+
+constexpr int SEL_THREADS = 1024;
+constexpr int SEL_WARPS = SEL_THREADS / 32;
+constexpr int SEL_SMEM_KEYS = 49152;  // rows up to this length keep their keys on chip
+constexpr int NBINS = 2048;
+
+__device__ __forceinline__ uint32_t float_to_key(float x) {
+  const uint32_t b = __float_as_uint(x);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// Exclusive prefix sum of one int per thread over the block; returns the prefix and
+// leaves the block total in *total_s after the second barrier.
+__device__ __forceinline__ int block_exclusive_scan(int x, int* warp_sums_s, int* total_s) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = x;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += y;
+  }
+  if (lane == 31) warp_sums_s[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_sums_s[lane];
+    int winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += y;
+    }
+    warp_sums_s[lane] = winc - w;  // exclusive
+    if (lane == 31) *total_s = winc;
+  }
+  __syncthreads();
+  return warp_sums_s[warp] + inc - x;
+}
+
+__global__ void __launch_bounds__(SEL_THREADS, 1)
+pool_topk_kernel(const float* __restrict__ vote, int n, int pool_kernel, int pool_type, int ksel,
+                 int32_t* __restrict__ out_idx, uint32_t* __restrict__ key_scratch) {
+  extern __shared__ uint32_t keys_smem[];
+  __shared__ int hist[NBINS];
+  __shared__ int warp_sums[SEL_WARPS];
+  __shared__ int scan_total;
+  __shared__ int sel_bin, sel_above;
+  __shared__ int wgt[SEL_WARPS], weq[SEL_WARPS];
+
+  const int row = blockIdx.x;
+  const float* vrow = vote + static_cast<size_t>(row) * n;
+  uint32_t* keys = key_scratch ? key_scratch + static_cast<size_t>(row) * n : keys_smem;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int r = pool_kernel >> 1;
+
+  // ---- 1. pooling
+  for (int j = threadIdx.x; j < n; j += SEL_THREADS) {
+    const int lo = max(0, j - r), hi = min(n - 1, j + r);
+    float p;
+    if (pool_type == 0) {
+      p = __ldg(vrow + lo);
+      for (int t = lo + 1; t <= hi; ++t) p = fmaxf(p, __ldg(vrow + t));
+    } else {
+      p = 0.f;
+      for (int t = lo; t <= hi; ++t) p += __ldg(vrow + t);
+      p = p / static_cast<float>(pool_kernel);
+    }
+    keys[j] = float_to_key(p);
+  }
+  __syncthreads();
+
+  // ---- 2. radix select of the ksel-th largest key
+  uint32_t prefix = 0, mask = 0;
+  int krem = ksel;
+  const int n_round = (n + 31) & ~31;
+#pragma unroll 1
+  for (int pass = 0; pass < 3; ++pass) {
+    const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+    const int nb = pass == 2 ? 1024 : 2048;
+    const uint32_t dmask = nb - 1;
+    for (int b = threadIdx.x; b < NBINS; b += SEL_THREADS) hist[b] = 0;
+    __syncthreads();
+    for (int base = warp * 32; base < n_round; base += SEL_THREADS) {
+      const int j = base + lane;
+      uint32_t key = 0;
+      bool live = false;
+      if (j < n) {
+        key = keys[j];
+        live = (key & mask) == prefix;
+      }
+      // lanes that do not take part get a value no other lane has
+      const uint32_t dg = live ? ((key >> shift) & dmask) : (0x80000000u | lane);
+      const uint32_t peers = __match_any_sync(0xffffffffu, dg);
+      if (live && lane == __ffs(peers) - 1) atomicAdd(&hist[dg], __popc(peers));
+    }
+    __syncthreads();
+    // walk the bins from the top: thread t owns bins nb-1-2t and nb-2-2t
+    int c0 = 0, c1 = 0;
+    const int b0 = nb - 1 - 2 * static_cast<int>(threadIdx.x);
+    if (b0 >= 0) c0 = hist[b0];
+    if (b0 - 1 >= 0) c1 = hist[b0 - 1];
+    const int before = block_exclusive_scan(c0 + c1, warp_sums, &scan_total);
+    if (c0 > 0 && before < krem && krem <= before + c0) {
+      sel_bin = b0;
+      sel_above = before;
+    } else if (c1 > 0 && before + c0 < krem && krem <= before + c0 + c1) {
+      sel_bin = b0 - 1;
+      sel_above = before + c0;
+    }
+    __syncthreads();
+    prefix |= static_cast<uint32_t>(sel_bin) << shift;
+    mask |= dmask << shift;
+    krem -= sel_above;
+    __syncthreads();
+  }
+  const uint32_t T = prefix;  // key of the ksel-th largest element
+  const int need_eq = krem;   // how many elements equal to T are kept (lowest positions)
+
+  // ---- 3. ordered compaction; warp w owns positions [w*span, (w+1)*span)
+  const int span = (((n + SEL_WARPS - 1) / SEL_WARPS) + 31) & ~31;
+  const int w_lo = warp * span;
+  const int w_hi = min(n, w_lo + span);
+  int cg = 0, ce = 0;
+  for (int base = w_lo; base < w_hi; base += 32) {
+    const int j = base + lane;
+    const uint32_t key = (j < w_hi) ? keys[j] : 0u;
+    cg += __popc(__ballot_sync(0xffffffffu, j < w_hi && key > T));
+    ce += __popc(__ballot_sync(0xffffffffu, j < w_hi && key == T));
+  }
+  if (lane == 0) {
+    wgt[warp] = cg;
+    weq[warp] = ce;
+  }
+  __syncthreads();
+  int gt_before = 0, eq_before = 0;
+  for (int w = 0; w < warp; ++w) {
+    gt_before += wgt[w];
+    eq_before += weq[w];
+  }
+  int out_pos = gt_before + min(eq_before, need_eq);
+  int32_t* orow = out_idx + static_cast<size_t>(row) * ksel;
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  for (int base = w_lo; base < w_hi; base += 32) {
+    const int j = base + lane;
+    const uint32_t key = (j < w_hi) ? keys[j] : 0u;
+    const bool gt = j < w_hi && key > T;
+    const bool eq = j < w_hi && key == T;
+    const uint32_t be = __ballot_sync(0xffffffffu, eq);
+    const bool take = gt || (eq && (eq_before + __popc(be & lt_mask)) < need_eq);
+    const uint32_t bt = __ballot_sync(0xffffffffu, take);
+    if (take) orow[out_pos + __popc(bt & lt_mask)] = j;
+    out_pos += __popc(bt);
+    eq_before += __popc(be);
+  }
+}
+
+__global__ void iota_kernel(int32_t* out, int rows, int n, int row_stride) {
+  const long long total = static_cast<long long>(rows) * n;
+  for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
+       i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const int rw = static_cast<int>(i / n);
+    const int j = static_cast<int>(i - static_cast<long long>(rw) * n);
+    out[static_cast<size_t>(rw) * row_stride + j] = j;
+  }
+}
+
+}  // namespace
+
+bool select_needs_scratch(int n) { return n > SEL_SMEM_KEYS; }
+
+cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel, int pool_type,
+                             int ksel, int32_t* out_idx, float* pooled_scratch,
+                             cudaStream_t stream, int* launches) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(pool_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         SEL_SMEM_KEYS * 4);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  const bool scratch = select_needs_scratch(n);
+  const size_t dyn = scratch ? 0 : static_cast<size_t>(n) * 4;
+  pool_topk_kernel<<<rows, SEL_THREADS, dyn, stream>>>(
+      vote, n, pool_kernel, pool_type, ksel, out_idx,
+      scratch ? reinterpret_cast<uint32_t*>(pooled_scratch) : nullptr);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_iota_idx(int32_t* out_idx, int rows, int n, int row_stride, cudaStream_t stream,
+                            int* launches) {
+  if (n <= 0) return cudaSuccess;
+  const long long total = static_cast<long long>(rows) * n;
+  int blocks = static_cast<int>((total + 255) / 256 < 1184 ? (total + 255) / 256 : 1184);
+  iota_kernel<<<blocks, 256, 0, stream>>>(out_idx, rows, n, row_stride);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
+}  // namespace snapkv
