@@ -75,7 +75,8 @@ __device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity) {
   }
 }
 
-template <int D, bool VOTE>
+// NCH = npad / 32: how many 32-column chunks of the accumulator a thread reads per tile.
+template <int D, bool VOTE, int NCH>
 __global__ void __launch_bounds__(THREADS, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
              const ScoreArgs a) {
@@ -232,42 +233,55 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       const int jmax = min(a.L - 1, a.n + i);
       float m2 = -INFINITY;  // running max, log2 domain
       float l = 0.f;         // running sum of exp2(x - m2)
-      const int nch = a.npad >> 5;
       for (int it = wg; it < nt; it += 2) {
         const int buf = it & (NBUF - 1);
         const uint32_t ub = (it / NBUF) & 1;
         if (!mbar_wait_warp(bar_tf(buf), ub, abort_s, WAIT_EPI_TMEM_FULL)) break;
         tc_fence_after();
         const int key0 = tile_of(it) * TILE_KEYS;
-        const bool need_mask = key0 + TILE_KEYS - 1 > a.n;
-        for (int ch = 0; ch < nch; ++ch) {
-          float v[32];
-          tmem_ld32(tmem_base + lane_sel + buf * 128 + rep * a.npad + ch * 32, v);
-          tmem_wait_ld();
-          if (need_mask) {
-            const int kb = key0 + rep * a.npad + ch * 32;
+        // the whole slice of this thread's row: NCH * 32 key columns
+        float v[NCH][32];
+        const uint32_t taddr = tmem_base + lane_sel + buf * 128 + rep * (NCH * 32);
 #pragma unroll
-            for (int c = 0; c < 32; ++c) v[c] = (kb + c <= jmax) ? v[c] : -INFINITY;
-          }
-          float cmax = v[0];
-#pragma unroll
-          for (int c = 1; c < 32; ++c) cmax = fmaxf(cmax, v[c]);
-          const float mnew = fmaxf(fmaxf(cmax * a.c2, m2), -1e30f);
-          l *= ex2_approx(m2 - mnew);
-          float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-          for (int c = 0; c < 32; c += 4) {
-            s0 += ex2_approx(fmaf(v[c + 0], a.c2, -mnew));
-            s1 += ex2_approx(fmaf(v[c + 1], a.c2, -mnew));
-            s2 += ex2_approx(fmaf(v[c + 2], a.c2, -mnew));
-            s3 += ex2_approx(fmaf(v[c + 3], a.c2, -mnew));
-          }
-          l += (s0 + s1) + (s2 + s3);
-          m2 = mnew;
-        }
+        for (int ch = 0; ch < NCH; ++ch) tmem_ld32(taddr + ch * 32, v[ch]);
+        tmem_wait_ld();
+        // the accumulator is in registers now: hand the buffer back to the MMA warp
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_te(buf));
+        if (key0 + TILE_KEYS - 1 > a.n) {  // tile touches the window or the end of the prompt
+          const int kb = key0 + rep * (NCH * 32);
+#pragma unroll
+          for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+            for (int c = 0; c < 32; ++c)
+              v[ch][c] = (kb + ch * 32 + c <= jmax) ? v[ch][c] : -INFINITY;
+        }
+        float c0 = v[0][0], c1 = v[0][1], c2m = v[0][2], c3 = v[0][3];
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+          for (int c = (ch == 0 ? 4 : 0); c < 32; c += 4) {
+            c0 = fmaxf(c0, v[ch][c + 0]);
+            c1 = fmaxf(c1, v[ch][c + 1]);
+            c2m = fmaxf(c2m, v[ch][c + 2]);
+            c3 = fmaxf(c3, v[ch][c + 3]);
+          }
+        const float cmax = fmaxf(fmaxf(c0, c1), fmaxf(c2m, c3));
+        const float mnew = fmaxf(fmaxf(cmax * a.c2, m2), -1e30f);
+        l *= ex2_approx(m2 - mnew);
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+          for (int c = 0; c < 32; c += 4) {
+            s0 += ex2_approx(fmaf(v[ch][c + 0], a.c2, -mnew));
+            s1 += ex2_approx(fmaf(v[ch][c + 1], a.c2, -mnew));
+            s2 += ex2_approx(fmaf(v[ch][c + 2], a.c2, -mnew));
+            s3 += ex2_approx(fmaf(v[ch][c + 3], a.c2, -mnew));
+          }
+        l += (s0 + s1) + (s2 + s3);
+        m2 = mnew;
       }
       part_s[(wg * 4 + q) * 32 + lane] = make_float2(m2, l);
       named_bar_sync(1, EPI_THREADS);
@@ -314,6 +328,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     } else {
       // ---------------------------------------------------------- votes
       const bool w16 = (a.W & 15) == 0;
+      const int gpw = a.W >> 4;  // 16-column groups per head (when W is a multiple of 16)
       for (int it = wg; it < nt; it += 2) {
         const int buf = it & (NBUF - 1);
         const uint32_t ub = (it / NBUF) & 1;
@@ -321,39 +336,55 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         tc_fence_after();
         const int j = tile_of(it) * TILE_KEYS + 32 * q + lane;
         const uint32_t taddr = tmem_base + lane_sel + buf * 128;
+        // this key's logits against every window row of the unit
+        float v[NCH][32];
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) tmem_ld32(taddr + ch * 32, v[ch]);
+        tmem_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_te(buf));
         if (w16) {
-          const int cpw = a.W >> 4;
-          for (int hl = 0; hl < a.hpu; ++hl) {
-            float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
-            for (int cc = 0; cc < cpw; ++cc) {
-              const int col = hl * a.W + cc * 16;
-              float v[16];
-              tmem_ld16(taddr + col, v);
-              tmem_wait_ld();
-              const float4* nl = reinterpret_cast<const float4*>(lse_s + col);
+          // exp2(s * c2 - lse2) summed over each group of 16 columns, then groups -> heads
+          float g16[NCH * 2];
+#pragma unroll
+          for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+              const float4* nl = reinterpret_cast<const float4*>(lse_s + ch * 32 + hf * 16);
+              float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
               for (int t4 = 0; t4 < 4; ++t4) {
                 const float4 z = nl[t4];
-                acc0 += ex2_approx(fmaf(v[4 * t4 + 0], a.c2, z.x));
-                acc1 += ex2_approx(fmaf(v[4 * t4 + 1], a.c2, z.y));
-                acc2 += ex2_approx(fmaf(v[4 * t4 + 2], a.c2, z.z));
-                acc3 += ex2_approx(fmaf(v[4 * t4 + 3], a.c2, z.w));
+                a0 += ex2_approx(fmaf(v[ch][hf * 16 + 4 * t4 + 0], a.c2, z.x));
+                a1 += ex2_approx(fmaf(v[ch][hf * 16 + 4 * t4 + 1], a.c2, z.y));
+                a2 += ex2_approx(fmaf(v[ch][hf * 16 + 4 * t4 + 2], a.c2, z.z));
+                a3 += ex2_approx(fmaf(v[ch][hf * 16 + 4 * t4 + 3], a.c2, z.w));
               }
+              g16[ch * 2 + hf] = (a0 + a1) + (a2 + a3);
             }
-            if (j < a.n)
-              a.vote[static_cast<size_t>(hq0 + hl) * a.n + j] = (acc0 + acc1) + (acc2 + acc3);
+          int hl = 0, left = gpw;
+          float acc = 0.f;
+#pragma unroll
+          for (int gi = 0; gi < NCH * 2; ++gi) {
+            acc += g16[gi];
+            if (--left == 0) {
+              if (hl < a.hpu && j < a.n) a.vote[static_cast<size_t>(hq0 + hl) * a.n + j] = acc;
+              acc = 0.f;
+              left = gpw;
+              ++hl;
+            }
           }
         } else {
           int hl = 0, left = a.W;
           float acc = 0.f;
-          for (int col0 = 0; col0 < a.ncols; col0 += 16) {
-            float v[16];
-            tmem_ld16(taddr + col0, v);
-            tmem_wait_ld();
 #pragma unroll
-            for (int t = 0; t < 16; ++t) {
-              if (col0 + t < a.ncols) {
-                acc += ex2_approx(fmaf(v[t], a.c2, lse_s[col0 + t]));
+          for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const int col = ch * 32 + c;
+              if (col < a.ncols) {
+                acc += ex2_approx(fmaf(v[ch][c], a.c2, lse_s[col]));
                 if (--left == 0) {
                   if (j < a.n) a.vote[static_cast<size_t>(hq0 + hl) * a.n + j] = acc;
                   acc = 0.f;
@@ -362,11 +393,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                 }
               }
             }
-          }
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_te(buf));
       }
     }
   }
@@ -413,17 +440,17 @@ bool encode_map(CUtensorMap* m, const void* base, int rank, const cuuint64_t* di
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D>
+template <int D, int NCH>
 cudaError_t run_passes(const CUtensorMap& tmK, const CUtensorMap& tmQ, ScoreArgs a,
                        const ScorePlan& p, cudaStream_t stream, int* launches) {
   static bool attr_done = false;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(score_kernel<D, false>,
+    cudaError_t e = cudaFuncSetAttribute(score_kernel<D, false, NCH>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          Smem<D>::DYN_BYTES);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(score_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             Smem<D>::DYN_BYTES);
+    e = cudaFuncSetAttribute(score_kernel<D, true, NCH>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::DYN_BYTES);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
@@ -432,11 +459,11 @@ cudaError_t run_passes(const CUtensorMap& tmK, const CUtensorMap& tmQ, ScoreArgs
     a.unit0 = u0;
     a.tiles = p.tiles_stats;
     a.chunks = p.chunks_stats;
-    score_kernel<D, false><<<dim3(p.chunks_stats, nu), THREADS, Smem<D>::DYN_BYTES, stream>>>(
+    score_kernel<D, false, NCH><<<dim3(p.chunks_stats, nu), THREADS, Smem<D>::DYN_BYTES, stream>>>(
         tmK, tmQ, a);
     a.tiles = p.tiles_vote;
     a.chunks = p.chunks_vote;
-    score_kernel<D, true><<<dim3(p.chunks_vote, nu), THREADS, Smem<D>::DYN_BYTES, stream>>>(
+    score_kernel<D, true, NCH><<<dim3(p.chunks_vote, nu), THREADS, Smem<D>::DYN_BYTES, stream>>>(
         tmK, tmQ, a);
     *launches += 2;
   }
@@ -522,8 +549,15 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq
   a.counters = counters;
   a.status = status;
   a.vote = vote;
-  if (d == 64) return run_passes<64>(tmK, tmQ, a, plan, stream, launches);
-  return run_passes<128>(tmK, tmQ, a, plan, stream, launches);
+  const int nch = plan.npad >> 5;
+  if (d == 64) {
+    if (nch == 1) return run_passes<64, 1>(tmK, tmQ, a, plan, stream, launches);
+    if (nch == 2) return run_passes<64, 2>(tmK, tmQ, a, plan, stream, launches);
+    return run_passes<64, 4>(tmK, tmQ, a, plan, stream, launches);
+  }
+  if (nch == 1) return run_passes<128, 1>(tmK, tmQ, a, plan, stream, launches);
+  if (nch == 2) return run_passes<128, 2>(tmK, tmQ, a, plan, stream, launches);
+  return run_passes<128, 4>(tmK, tmQ, a, plan, stream, launches);
 }
 
 }  // namespace snapkv

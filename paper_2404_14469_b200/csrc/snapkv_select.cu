@@ -1,5 +1,8 @@
 // Pooling and per-head top-k (Listing 1's pool1d and topk; Eq. 2), one CTA per row.
 //
+// Two kernels: a fast one for rows that fit in shared memory (below) and this generic
+// one, which also handles rows of any length through global scratch.
+//
 //  1. pooled[j] = max or mean of vote[j-r .. j+r] (stride 1, same length; the mean
 //     divides by pool_kernel, positions outside the row count as zero), turned into a
 //     32-bit key whose unsigned order is the float order.  Keys stay in shared memory
@@ -171,6 +174,153 @@ pool_topk_kernel(const float* __restrict__ vote, int n, int pool_kernel, int poo
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// Fast path for rows that fit in shared memory and pooling radii up to RMAX.
+// Thread t owns the EPT consecutive positions [t*EPT, (t+1)*EPT): pooling is a sliding
+// window over registers, histogram updates are run-length aggregated (pooled neighbours
+// fall into the same bin), and the ordered compaction is a single block scan.  Keys sit
+// in shared memory at slot j + j/32, which keeps the strided per-thread sweeps free of
+// bank conflicts.  The first histogram pass bins (key - min) >> shift with the shift
+// chosen from the row's key range, so the bins are spread over the values that occur.
+__device__ __forceinline__ int key_slot(int j) { return j + (j >> 5); }
+
+template <int RMAX>
+__global__ void __launch_bounds__(SEL_THREADS, 1)
+pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_type, int ept,
+                      int ksel, int32_t* __restrict__ out_idx) {
+  extern __shared__ uint32_t keys[];
+  __shared__ int hist[NBINS];
+  __shared__ int warp_sums[SEL_WARPS];
+  __shared__ int scan_total;
+  __shared__ int sel_bin, sel_above;
+  __shared__ uint32_t red_min[SEL_WARPS], red_max[SEL_WARPS];
+
+  const int row = blockIdx.x;
+  const float* vrow = vote + static_cast<size_t>(row) * n;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int base = threadIdx.x * ept;
+
+  // ---- 1. pooling over a rolling register window
+  uint32_t kmin = 0xffffffffu, kmax = 0u;
+  {
+    float w[2 * RMAX + 8];
+#pragma unroll
+    for (int i = 0; i < 2 * RMAX; ++i) {
+      const int j = base - RMAX + i;
+      w[i] = (j >= 0 && j < n) ? __ldg(vrow + j) : 0.f;
+    }
+    for (int sb = 0; sb < ept; sb += 8) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int j = base + sb + RMAX + i;
+        w[2 * RMAX + i] = (j < n) ? __ldg(vrow + j) : 0.f;
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        float p = 0.f;  // votes are >= 0: zero is neutral for max and is the avg padding
+#pragma unroll
+        for (int t = 0; t <= 2 * RMAX; ++t) {
+          const int off = t - RMAX;
+          if (off >= -r && off <= r) p = (pool_type == 0) ? fmaxf(p, w[i + t]) : p + w[i + t];
+        }
+        const int j = base + sb + i;
+        uint32_t key = 0u;  // positions past the row end rank below every real key
+        if (j < n) {
+          key = float_to_key(p);
+          kmin = min(kmin, key);
+          kmax = max(kmax, key);
+        }
+        keys[key_slot(j)] = key;
+      }
+#pragma unroll
+      for (int i = 0; i < 2 * RMAX; ++i) w[i] = w[i + 8];
+    }
+  }
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if (lane == 0) {
+    red_min[warp] = kmin;
+    red_max[warp] = kmax;
+  }
+  __syncthreads();
+  kmin = red_min[lane];
+  kmax = red_max[lane];
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+
+  // ---- 2. threshold: histogram passes over an ever narrower key range [lo, lo + width)
+  uint32_t lo = kmin;
+  int krem = ksel;
+  uint32_t T = kmin;
+  if (kmax != kmin) {
+    const uint32_t range = kmax - kmin;
+    int shift = 32 - __clz(range) - 11;
+    if (shift < 0) shift = 0;
+    uint32_t width_m1 = range;  // candidates are keys with key - lo <= width_m1
+#pragma unroll 1
+    for (;;) {
+      for (int b = threadIdx.x; b < NBINS; b += SEL_THREADS) hist[b] = 0;
+      __syncthreads();
+      int cur = -1, cnt = 0;
+      for (int i = 0; i < ept; ++i) {
+        const uint32_t key = keys[key_slot(base + i)];
+        const uint32_t rel = key - lo;
+        if (key >= lo && rel <= width_m1) {
+          const int b = static_cast<int>(rel >> shift);
+          if (b != cur) {
+            if (cnt) atomicAdd(&hist[cur], cnt);
+            cur = b;
+            cnt = 0;
+          }
+          ++cnt;
+        }
+      }
+      if (cnt) atomicAdd(&hist[cur], cnt);
+      __syncthreads();
+      int c0 = 0, c1 = 0;
+      const int b0 = NBINS - 1 - 2 * static_cast<int>(threadIdx.x);
+      if (b0 >= 0) c0 = hist[b0];
+      if (b0 - 1 >= 0) c1 = hist[b0 - 1];
+      const int before = block_exclusive_scan(c0 + c1, warp_sums, &scan_total);
+      if (c0 > 0 && before < krem && krem <= before + c0) {
+        sel_bin = b0;
+        sel_above = before;
+      } else if (c1 > 0 && before + c0 < krem && krem <= before + c0 + c1) {
+        sel_bin = b0 - 1;
+        sel_above = before + c0;
+      }
+      __syncthreads();
+      krem -= sel_above;
+      lo += static_cast<uint32_t>(sel_bin) << shift;
+      const int done = (shift == 0);
+      __syncthreads();
+      if (done) break;
+      width_m1 = (1u << shift) - 1u;
+      shift = shift > 11 ? shift - 11 : 0;
+    }
+    T = lo;
+  }
+  const int need_eq = krem;
+
+  // ---- 3. ordered compaction
+  int cg = 0, ce = 0;
+  for (int i = 0; i < ept; ++i) {
+    const uint32_t key = keys[key_slot(base + i)];
+    cg += key > T;
+    ce += key == T;
+  }
+  const int packed = block_exclusive_scan((cg << 16) | ce, warp_sums, &scan_total);
+  int eq_before = packed & 0xffff;
+  int out_pos = (packed >> 16) + min(eq_before, need_eq);
+  int32_t* orow = out_idx + static_cast<size_t>(row) * ksel;
+  if (cg + ce > 0) {
+    for (int i = 0; i < ept; ++i) {
+      const uint32_t key = keys[key_slot(base + i)];
+      if (key > T || (key == T && eq_before++ < need_eq)) orow[out_pos++] = base + i;
+    }
+  }
+}
+
 __global__ void iota_kernel(int32_t* out, int rows, int n, int row_stride) {
   const long long total = static_cast<long long>(rows) * n;
   for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
@@ -183,6 +333,9 @@ __global__ void iota_kernel(int32_t* out, int rows, int n, int row_stride) {
 
 }  // namespace
 
+static inline int key_slot_host(int j) { return j + (j >> 5); }
+constexpr int FAST_SMEM_BYTES = (SEL_SMEM_KEYS + SEL_SMEM_KEYS / 32 + 64) * 4;
+
 bool select_needs_scratch(int n) { return n > SEL_SMEM_KEYS; }
 
 cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel, int pool_type,
@@ -193,7 +346,26 @@ cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel
     cudaError_t e = cudaFuncSetAttribute(pool_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          SEL_SMEM_KEYS * 4);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(pool_topk_fast_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             FAST_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(pool_topk_fast_kernel<7>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             FAST_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
     attr_done = true;
+  }
+  const int r = pool_kernel >> 1;
+  if (n <= SEL_SMEM_KEYS && r <= 7) {
+    const int ept = (((n + SEL_THREADS - 1) / SEL_THREADS) + 7) & ~7;
+    const int words = key_slot_host(SEL_THREADS * ept) + 1;
+    if (r <= 3)
+      pool_topk_fast_kernel<3><<<rows, SEL_THREADS, words * 4, stream>>>(vote, n, r, pool_type, ept,
+                                                                       ksel, out_idx);
+    else
+      pool_topk_fast_kernel<7><<<rows, SEL_THREADS, words * 4, stream>>>(vote, n, r, pool_type, ept,
+                                                                       ksel, out_idx);
+    *launches += 1;
+    return cudaGetLastError();
   }
   const bool scratch = select_needs_scratch(n);
   const size_t dyn = scratch ? 0 : static_cast<size_t>(n) * 4;
