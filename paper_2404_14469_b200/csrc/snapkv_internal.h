@@ -10,6 +10,7 @@ constexpr int TILE_KEYS = 128;      // keys per MMA tile
 constexpr int MAX_COLS = 128;       // window-query columns handled by one unit
 constexpr int STATUS_BYTES = 256;   // status block at the start of every workspace
 constexpr int SM_COUNT_HINT = 148;  // B200
+constexpr int MAX_GRID = 192;       // the scoring kernel runs one CTA per SM, at most this many
 
 // Codes stored in the workspace status block's second word when a wait gives up.
 enum WaitCode {
@@ -20,6 +21,7 @@ enum WaitCode {
   WAIT_EPI_TMEM_FULL = 4,
   WAIT_Q_FULL = 5,
   WAIT_DRAIN = 6,
+  WAIT_UNIT_STATS = 7,
 };
 
 // How the scoring passes split the work.  A "unit" is one (batch, KV head, head
@@ -34,12 +36,13 @@ struct ScorePlan {
   int tiles_stats;  // ceil(L / TILE_KEYS): the normaliser covers every key
   int tiles_vote;   // ceil(n / TILE_KEYS): votes exist for prefix keys only
   int units_per_wave;
-  int chunks_stats; // CTAs per unit in the statistics pass
-  int chunks_vote;  // CTAs per unit in the vote pass
+  int nwaves;
+  int maxseg;       // partial-statistics slots per unit
+  int pipelined;    // phase order S0 S1 V0 S2 V1 ... (1) or S0 V0 S1 V1 ... (0)
 };
 
 struct WorkspaceLayout {
-  size_t off_status, off_counters, off_partials, off_lse, off_vote, off_pooled, total;
+  size_t off_status, off_counters, off_partials, off_vote, off_pooled, total;
 };
 
 bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* plan);
@@ -50,7 +53,7 @@ bool select_needs_scratch(int n);
 // Enqueue both scoring passes.  `vote` is fp32 [B*Hq, n].
 cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv, int L,
                                  int d, int W, const ScorePlan& plan, float* vote, int* status,
-                                 int* counters, float2* partials, float* lse2, cudaStream_t stream,
+                                 int* counters, float2* partials, cudaStream_t stream,
                                  int* launches);
 
 // Pool + top-k over `rows` rows of fp32 votes.  `pooled_scratch` (fp32 [rows, n]) is

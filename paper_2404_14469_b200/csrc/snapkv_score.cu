@@ -1,22 +1,31 @@
 // Window scoring (Eq. 1; Listing 1's compute_attn and the sum over the window):
 //   vote[h, j] = sum_i softmax_i(q_i . k / sqrt(d))[j],  j in [0, n)
-// computed in two tensor-core passes over K.
+// computed in two tensor-core passes over K inside ONE persistent kernel.
 //
-//  pass 1 (statistics)  S^T tile = Q_rep[128 x d] . K_tile[128 x d]^T : window rows on
+//  pass S (statistics)  S^T tile = Q_rep[128 x d] . K_tile[128 x d]^T : window rows on
 //      TMEM lanes, keys on columns.  Each thread owns one window row and keeps a running
 //      (max, sum of exp) over the keys it sees: an online softmax without shuffles.
 //      When the unit has fewer than 128 window rows the rows are replicated along M and
 //      each replica takes a different slice of the tile's keys, so all four epilogue
-//      warps of a warpgroup stay busy.  The last CTA of a unit to finish merges the
-//      partial (max, sum) pairs into one log2-sum-exp per window row.
-//  pass 2 (votes)       S tile = K_tile[128 x d] . Q[ncols x d]^T : keys on TMEM lanes,
-//      window rows on columns.  Each thread owns one key and adds exp2(s*c - lse) over
-//      the W columns of each head: the sum over the window is a serial add per thread.
+//      warps of a warpgroup stay busy.  Each CTA publishes one (max, sum) pair per window
+//      row for the keys it saw and bumps the unit's counter.
+//  pass V (votes)       S tile = K_tile[128 x d] . Q[ncols x d]^T : keys on TMEM lanes,
+//      window rows on columns.  Once the unit's counter shows that every partial has been
+//      published, the CTA merges them into one log2-sum-exp per window row; then each
+//      thread owns one key and adds exp2(s*c - lse) over the W columns of each head: the
+//      sum over the window is a serial add per thread.
 //
-// Both passes share one warp-specialised skeleton: warp 0 issues TMA loads of K tiles
-// into a ring of shared-memory stages, warp 1 issues tcgen05.mma into four TMEM
-// accumulator buffers, warps 2-9 (two warpgroups, alternating tiles) read the
-// accumulators back with tcgen05.ld and do the fp32 softmax arithmetic.
+// Units (batch, KV head, head sub-group) are grouped into waves small enough for L2; the
+// kernel walks the phases  S(0), S(1), V(0), S(2), V(1), ...  so that the second sweep
+// over a wave's keys is served by L2 and the partials a vote phase needs were published
+// a whole phase earlier.  Within a phase the wave's tiles are split evenly over the CTAs.
+// One CTA per SM, launched cooperatively (all CTAs are resident, so waiting on another
+// CTA's partials cannot starve it).
+//
+// Warp roles: warp 0 issues TMA loads (K tiles into a ring of stages, Q per work item
+// into two buffers), warp 1 issues tcgen05.mma into four TMEM accumulator buffers, warps
+// 2-9 (two warpgroups, alternating tiles) read the accumulators back with tcgen05.ld and
+// do the fp32 softmax arithmetic.
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <math.h>
@@ -40,11 +49,13 @@ struct ScoreArgs {
   int L, n, W;
   int hpu, ncols, npad;
   int sub_per_kv, g;
-  int tiles, chunks, unit0;
-  float c2;  // log2(e) / sqrt(d)
-  float2* partials;
-  float* lse2;
-  int* counters;
+  int units, upw, nwaves;   // units per wave, number of waves
+  int T1, T2;               // tiles per unit in the statistics / vote pass
+  int maxseg;               // partial slots per unit
+  int pipelined;            // phase order S0 S1 V0 S2 V1 ... (else S0 V0 S1 V1 ...)
+  float c2;                 // log2(e) / sqrt(d)
+  float2* partials;         // [units][maxseg][MAX_COLS] (max, sum) in the log2 domain
+  int* counters;            // [units] published partials
   int* status;
   float* vote;
 };
@@ -54,13 +65,13 @@ struct Smem {
   static constexpr int SUBT = D / 64;
   static constexpr int Q_BYTES = SUBT * SUBTILE_BYTES;
   static constexpr int STAGE_BYTES = SUBT * SUBTILE_BYTES;
-  static constexpr int OFF_Q = 0;
-  static constexpr int OFF_K = Q_BYTES;
+  static constexpr int OFF_Q = 0;                            // two Q buffers
+  static constexpr int OFF_K = 2 * Q_BYTES;
   static constexpr int OFF_BAR = OFF_K + STAGES * STAGE_BYTES;
-  // barriers: full[STAGES], empty[STAGES], tf[NBUF], te[NBUF], qfull, drain
-  static constexpr int NBAR = 2 * STAGES + 2 * NBUF + 2;
-  static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;       // tmem ptr, abort, last flag
-  static constexpr int OFF_PART = OFF_MISC + 16;            // float2 [8][32]
+  // barriers: full[STAGES], empty[STAGES], tf[NBUF], te[NBUF], qfull[2], qempty[2], drain
+  static constexpr int NBAR = 2 * STAGES + 2 * NBUF + 5;
+  static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;       // tmem ptr, abort
+  static constexpr int OFF_PART = OFF_MISC + 24;            // float2 [8][32]
   static constexpr int OFF_LSE = OFF_PART + 8 * 32 * 8;     // float [128]
   static constexpr int TOTAL = OFF_LSE + 128 * 4;
   static constexpr int DYN_BYTES = TOTAL + 1024;            // slack for 1024-byte alignment
@@ -75,42 +86,102 @@ __device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity) {
   }
 }
 
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// One piece of work: tiles [t0, t1) of one unit in one pass.
+struct Item {
+  int unit, t0, t1, vote, slot, nseg;
+};
+
+// CTA `c` of `G` owns tiles [c*TT/G, (c+1)*TT/G) of a phase's TT tiles.
+__device__ __forceinline__ long long part_lo(long long c, long long TT, int G) { return c * TT / G; }
+// the CTA whose range contains tile x: the largest c with part_lo(c) <= x
+__device__ __forceinline__ int cta_of_tile(long long x, long long TT, int G) {
+  return static_cast<int>(((x + 1) * G + TT - 1) / TT) - 1;
+}
+
+// Calls f(item) for every work item of this CTA in schedule order; stops when f
+// returns false.  All three warp roles walk the same list.
+template <typename F>
+__device__ __forceinline__ void for_each_item(const ScoreArgs& a, int cta, int G, F&& f) {
+  const int nph = 2 * a.nwaves;
+  for (int p = 0; p < nph; ++p) {
+    int w, vote;
+    if (a.pipelined) {
+      if (p == 0) { w = 0; vote = 0; }
+      else if (p == nph - 1) { w = a.nwaves - 1; vote = 1; }
+      else if (p & 1) { w = (p + 1) >> 1; vote = 0; }
+      else { w = (p >> 1) - 1; vote = 1; }
+    } else {
+      w = p >> 1;
+      vote = p & 1;
+    }
+    const int u0 = w * a.upw;
+    const int nu = min(a.upw, a.units - u0);
+    const int T = vote ? a.T2 : a.T1;
+    const long long TT = static_cast<long long>(nu) * T;
+    const long long lo = part_lo(cta, TT, G), hi = part_lo(cta + 1, TT, G);
+    for (long long pos = lo; pos < hi;) {
+      const int ul = static_cast<int>(pos / T);
+      Item it;
+      it.unit = u0 + ul;
+      it.t0 = static_cast<int>(pos - static_cast<long long>(ul) * T);
+      it.t1 = static_cast<int>(min(static_cast<long long>(T), it.t0 + (hi - pos)));
+      it.vote = vote;
+      // where this CTA's partial of the unit goes / how many partials the unit gets:
+      // both follow from the statistics-pass partition of the unit's wave
+      const long long TT1 = static_cast<long long>(nu) * a.T1;
+      if (TT1 >= G) {  // every CTA has tiles: a unit's owners are consecutive CTAs
+        const int cfirst = cta_of_tile(static_cast<long long>(ul) * a.T1, TT1, G);
+        const int clast = cta_of_tile(static_cast<long long>(ul + 1) * a.T1 - 1, TT1, G);
+        it.slot = cta - cfirst;
+        it.nseg = clast - cfirst + 1;
+      } else {         // fewer tiles than CTAs: one tile per owner, one partial per tile
+        it.slot = it.t0;
+        it.nseg = a.T1;
+      }
+      pos += it.t1 - it.t0;
+      if (!f(it)) return;
+    }
+  }
+}
+
 // NCH = npad / 32: how many 32-column chunks of the accumulator a thread reads per tile.
-template <int D, bool VOTE, int NCH>
+template <int D, int NCH>
 __global__ void __launch_bounds__(THREADS, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
              const ScoreArgs a) {
   using SM = Smem<D>;
   constexpr int SUBT = SM::SUBT;
+  constexpr int NPAD = NCH * 32;
+  constexpr int REPS = 128 / NPAD;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
   const uint32_t sbase = smem_u32(smem);
-  const uint32_t q_s = sbase + SM::OFF_Q;
   const uint32_t k_s = sbase + SM::OFF_K;
   const uint32_t bar0 = sbase + SM::OFF_BAR;
+  auto q_s = [&](int b) { return sbase + SM::OFF_Q + b * SM::Q_BYTES; };
   auto bar_full = [&](int s) { return bar0 + 8u * s; };
   auto bar_empty = [&](int s) { return bar0 + 8u * (STAGES + s); };
   auto bar_tf = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
   auto bar_te = [&](int b) { return bar0 + 8u * (2 * STAGES + NBUF + b); };
-  const uint32_t bar_q = bar0 + 8u * (2 * STAGES + 2 * NBUF);
-  const uint32_t bar_drain = bar_q + 8u;
+  auto bar_qf = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 * NBUF + b); };
+  auto bar_qe = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 * NBUF + 2 + b); };
+  const uint32_t bar_drain = bar0 + 8u * (2 * STAGES + 2 * NBUF + 4);
   volatile uint32_t* tmem_ptr_s = reinterpret_cast<volatile uint32_t*>(smem + SM::OFF_MISC);
   volatile int* abort_s = reinterpret_cast<volatile int*>(smem + SM::OFF_MISC + 4);
-  volatile int* last_s = reinterpret_cast<volatile int*>(smem + SM::OFF_MISC + 8);
   float2* part_s = reinterpret_cast<float2*>(smem + SM::OFF_PART);
   float* lse_s = reinterpret_cast<float*>(smem + SM::OFF_LSE);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int chunk = blockIdx.x;
-  const int u = a.unit0 + blockIdx.y;          // unit
-  const int ukv = u / a.sub_per_kv;            // flat (batch, KV head)
-  const int sub = u - ukv * a.sub_per_kv;
-  const int hq0 = ukv * a.g + sub * a.hpu;     // first query head of the unit, flat over batch
-  const int t_begin = static_cast<int>((static_cast<long long>(chunk) * a.tiles) / a.chunks);
-  const int t_end = static_cast<int>((static_cast<long long>(chunk + 1) * a.tiles) / a.chunks);
-  const int nt = t_end - t_begin;
+  const int cta = blockIdx.x;
+  const int G = gridDim.x;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -121,67 +192,80 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       mbar_init(bar_tf(b), 1);
       mbar_init(bar_te(b), 4);
     }
-    mbar_init(bar_q, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_qf(b), 1);
+      mbar_init(bar_qe(b), 1);
+    }
     mbar_init(bar_drain, 1);
     *abort_s = 0;
-    *last_s = 0;
     mbar_fence_init();
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_ptr_s)), TMEM_COLS);
     tmem_relinquish();
   }
-  if (VOTE) {
-    // -lse2 of this unit's window rows, written by the statistics pass
-    if (threadIdx.x >= 64 && threadIdx.x < 64 + 128) {
-      const int c = threadIdx.x - 64;
-      lse_s[c] = (c < a.ncols) ? -__ldcg(a.lse2 + static_cast<size_t>(u) * MAX_COLS + c) : 0.f;
-    }
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_ptr_s;
 
-  // tile visited at iteration `it`: ascending in the statistics pass, descending in the
-  // vote pass (the tiles read last by pass 1 are the most likely to still be in L2)
-  auto tile_of = [&](int it) { return VOTE ? (t_end - 1 - it) : (t_begin + it); };
+  // tile visited at step k of an item: ascending, except that the sequential schedule
+  // sweeps the vote pass backwards (the keys read last are the likeliest to be in L2)
+  auto tile_of = [&](const Item& it, int k) {
+    return (it.vote && !a.pipelined) ? (it.t1 - 1 - k) : (it.t0 + k);
+  };
+  auto first_head = [&](int unit, int* ukv) {
+    *ukv = unit / a.sub_per_kv;
+    return *ukv * a.g + (unit - *ukv * a.sub_per_kv) * a.hpu;  // flat over the batch
+  };
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tmK);
       tma_prefetch_desc(&tmQ);
-      const int qrow0 = hq0 * a.W;
-      if (VOTE) {
-        mbar_expect_tx(bar_q, SUBT * a.npad * 128);
-        for (int sb = 0; sb < SUBT; ++sb)
-          tma_load_2d(q_s + sb * SUBTILE_BYTES, &tmQ, bar_q, sb * 64, qrow0);
-      } else {
-        mbar_expect_tx(bar_q, SUBT * 128 * 128);
-        const int reps = 128 / a.npad;
-        for (int rep = 0; rep < reps; ++rep)
+      int git = 0;      // tiles issued so far (ring position)
+      int nitem = 0;    // items started so far (Q buffer position)
+      for_each_item(a, cta, G, [&](const Item& it) {
+        int ukv;
+        const int qrow0 = first_head(it.unit, &ukv) * a.W;
+        const int qb = nitem & 1;
+        if (!mbar_wait_thread(bar_qe(qb), ((nitem >> 1) & 1) ^ 1, abort_s, WAIT_Q_FULL)) return false;
+        if (it.vote) {
+          mbar_expect_tx(bar_qf(qb), SUBT * NPAD * 128);
           for (int sb = 0; sb < SUBT; ++sb)
-            tma_load_2d(q_s + sb * SUBTILE_BYTES + rep * a.npad * 128, &tmQ, bar_q, sb * 64, qrow0);
-      }
-      int issued = 0;
-      for (int it = 0; it < nt; ++it) {
-        const int s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1;
-        if (!mbar_wait_thread(bar_empty(s), ph ^ 1, abort_s, WAIT_PRODUCER_EMPTY)) break;
-        mbar_expect_tx(bar_full(s), SM::STAGE_BYTES);
-        const int key0 = tile_of(it) * TILE_KEYS;
-        for (int sb = 0; sb < SUBT; ++sb)
-          tma_load_3d(k_s + s * SM::STAGE_BYTES + sb * SUBTILE_BYTES, &tmK, bar_full(s), sb * 64,
-                      key0, ukv);
-        issued = it + 1;
-      }
+            tma_load_2d(q_s(qb) + sb * SUBTILE_BYTES, &tmQ, bar_qf(qb), sb * 64, qrow0);
+        } else {
+          mbar_expect_tx(bar_qf(qb), SUBT * 128 * 128);
+          for (int rep = 0; rep < REPS; ++rep)
+            for (int sb = 0; sb < SUBT; ++sb)
+              tma_load_2d(q_s(qb) + sb * SUBTILE_BYTES + rep * NPAD * 128, &tmQ, bar_qf(qb),
+                          sb * 64, qrow0);
+        }
+        ++nitem;
+        const int nt = it.t1 - it.t0;
+        for (int k = 0; k < nt; ++k, ++git) {
+          const int s = git % STAGES;
+          const uint32_t ph = (git / STAGES) & 1;
+          if (!mbar_wait_thread(bar_empty(s), ph ^ 1, abort_s, WAIT_PRODUCER_EMPTY)) return false;
+          mbar_expect_tx(bar_full(s), SM::STAGE_BYTES);
+          const int key0 = tile_of(it, k) * TILE_KEYS;
+          for (int sb = 0; sb < SUBT; ++sb)
+            tma_load_3d(k_s + s * SM::STAGE_BYTES + sb * SUBTILE_BYTES, &tmK, bar_full(s), sb * 64,
+                        key0, ukv);
+        }
+        return true;
+      });
       if (*abort_s != 0) {
         // let every copy in flight land before the CTA's shared memory goes away
-        mbar_wait_drain(bar_q, 0);
+        for (int b = 0; b < 2; ++b) {
+          int last = -1;
+          for (int i = b; i < nitem; i += 2) last = i;
+          if (last >= 0) mbar_wait_drain(bar_qf(b), (last >> 1) & 1);
+        }
         for (int s = 0; s < STAGES; ++s) {
           int last = -1;
-          for (int it = s; it < issued; it += STAGES) last = it;
+          for (int i = s; i < git; i += STAGES) last = i;
           if (last >= 0) mbar_wait_drain(bar_full(s), (last / STAGES) & 1);
         }
       }
@@ -189,31 +273,40 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = VOTE ? umma_idesc_bf16(128, a.npad) : umma_idesc_bf16(128, 128);
-      bool ok = mbar_wait_thread(bar_q, 0, abort_s, WAIT_Q_FULL);
-      for (int it = 0; ok && it < nt; ++it) {
-        const int s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1;
-        const int buf = it & (NBUF - 1);
-        const uint32_t ub = (it / NBUF) & 1;
-        if (!mbar_wait_thread(bar_full(s), ph, abort_s, WAIT_MMA_FULL)) break;
-        if (!mbar_wait_thread(bar_te(buf), ub ^ 1, abort_s, WAIT_MMA_TMEM_EMPTY)) break;
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * 128;
+      const uint32_t idesc_s = umma_idesc_bf16(128, 128);
+      const uint32_t idesc_v = umma_idesc_bf16(128, NPAD);
+      int git = 0, nitem = 0;
+      for_each_item(a, cta, G, [&](const Item& it) {
+        const int qb = nitem & 1;
+        if (!mbar_wait_thread(bar_qf(qb), (nitem >> 1) & 1, abort_s, WAIT_Q_FULL)) return false;
+        ++nitem;
+        const int nt = it.t1 - it.t0;
+        for (int k = 0; k < nt; ++k, ++git) {
+          const int s = git % STAGES;
+          const uint32_t ph = (git / STAGES) & 1;
+          const int buf = git & (NBUF - 1);
+          const uint32_t ub = (git / NBUF) & 1;
+          if (!mbar_wait_thread(bar_full(s), ph, abort_s, WAIT_MMA_FULL)) return false;
+          if (!mbar_wait_thread(bar_te(buf), ub ^ 1, abort_s, WAIT_MMA_TMEM_EMPTY)) return false;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + buf * 128;
 #pragma unroll
-        for (int sb = 0; sb < SUBT; ++sb) {
+          for (int sb = 0; sb < SUBT; ++sb) {
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {
-            const uint64_t kd =
-                umma_desc_k128(k_s + s * SM::STAGE_BYTES + sb * SUBTILE_BYTES + kk * 32);
-            const uint64_t qd = umma_desc_k128(q_s + sb * SUBTILE_BYTES + kk * 32);
-            if (VOTE) tc_mma_bf16(d_tmem, kd, qd, idesc, (sb | kk) != 0);
-            else tc_mma_bf16(d_tmem, qd, kd, idesc, (sb | kk) != 0);
+            for (int kk = 0; kk < 4; ++kk) {
+              const uint64_t kd =
+                  umma_desc_k128(k_s + s * SM::STAGE_BYTES + sb * SUBTILE_BYTES + kk * 32);
+              const uint64_t qd = umma_desc_k128(q_s(qb) + sb * SUBTILE_BYTES + kk * 32);
+              if (it.vote) tc_mma_bf16(d_tmem, kd, qd, idesc_v, (sb | kk) != 0);
+              else tc_mma_bf16(d_tmem, qd, kd, idesc_s, (sb | kk) != 0);
+            }
           }
+          tc_commit(bar_empty(s));
+          tc_commit(bar_tf(buf));
         }
-        tc_commit(bar_empty(s));
-        tc_commit(bar_tf(buf));
-      }
+        tc_commit(bar_qe(qb));  // the item's MMAs are the last readers of its Q buffer
+        return true;
+      });
       if (*abort_s != 0) {
         tc_commit(bar_drain);
         mbar_wait_drain(bar_drain, 0);
@@ -221,120 +314,157 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     }
   } else {
     // ------------------------------------------------------------ softmax warps
-    const int e = warp - 2;
-    const int wg = e >> 2;
+    const int wg = (warp - 2) >> 2;
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     const uint32_t lane_sel = static_cast<uint32_t>(32 * q) << 16;
-    if (!VOTE) {
-      const int rrow = 32 * q + lane;
-      const int rep = rrow / a.npad;
-      const int qcol = rrow - rep * a.npad;
-      const int i = qcol % a.W;
-      const int jmax = min(a.L - 1, a.n + i);
-      float m2 = -INFINITY;  // running max, log2 domain
-      float l = 0.f;         // running sum of exp2(x - m2)
-      for (int it = wg; it < nt; it += 2) {
-        const int buf = it & (NBUF - 1);
-        const uint32_t ub = (it / NBUF) & 1;
-        if (!mbar_wait_warp(bar_tf(buf), ub, abort_s, WAIT_EPI_TMEM_FULL)) break;
-        tc_fence_after();
-        const int key0 = tile_of(it) * TILE_KEYS;
-        // the whole slice of this thread's row: NCH * 32 key columns
-        float v[NCH][32];
-        const uint32_t taddr = tmem_base + lane_sel + buf * 128 + rep * (NCH * 32);
+    const int tid = threadIdx.x - 64;
+    const int rrow = 32 * q + lane;  // TMEM lane
+    const int rep = rrow / NPAD;
+    const int qcol = rrow - rep * NPAD;
+    const int jmax = min(a.L - 1, a.n + (qcol % a.W));  // last key window row qcol % W sees
+    const bool w16 = (a.W & 15) == 0;
+    const int gpw = a.W >> 4;  // 16-column groups per head (when W is a multiple of 16)
+    int git = 0;
+    // Once a wait has given up (here or in another role) this warp stops touching TMEM
+    // and barriers of the pipeline but still walks every item, so that all eight warps
+    // keep meeting at the named barriers and reach the end of the kernel together.
+    bool dead = false;
+    for_each_item(a, cta, G, [&](const Item& it) {
+      const int nt = it.t1 - it.t0;
+      int ukv;
+      const int hq0 = first_head(it.unit, &ukv);
+      if (!it.vote) {
+        // ---------------------------------------------------------- statistics
+        float m2 = -INFINITY;  // running max, log2 domain
+        float l = 0.f;         // running sum of exp2(x - m2)
+        for (int k = 0; k < nt; ++k, ++git) {
+          if ((git & 1) != wg || dead) continue;
+          const int buf = git & (NBUF - 1);
+          const uint32_t ub = (git / NBUF) & 1;
+          if (!mbar_wait_warp(bar_tf(buf), ub, abort_s, WAIT_EPI_TMEM_FULL)) {
+            dead = true;
+            continue;
+          }
+          tc_fence_after();
+          const int key0 = tile_of(it, k) * TILE_KEYS;
+          // the whole slice of this thread's row: NPAD key columns
+          float v[NCH][32];
+          const uint32_t taddr = tmem_base + lane_sel + buf * 128 + rep * NPAD;
 #pragma unroll
-        for (int ch = 0; ch < NCH; ++ch) tmem_ld32(taddr + ch * 32, v[ch]);
-        tmem_wait_ld();
-        // the accumulator is in registers now: hand the buffer back to the MMA warp
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_te(buf));
-        if (key0 + TILE_KEYS - 1 > a.n) {  // tile touches the window or the end of the prompt
-          const int kb = key0 + rep * (NCH * 32);
+          for (int ch = 0; ch < NCH; ++ch) tmem_ld32(taddr + ch * 32, v[ch]);
+          tmem_wait_ld();
+          // the accumulator is in registers now: hand the buffer back to the MMA warp
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_te(buf));
+          if (key0 + TILE_KEYS - 1 > a.n) {  // tile touches the window or the prompt's end
+            const int kb = key0 + rep * NPAD;
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                v[ch][c] = (kb + ch * 32 + c <= jmax) ? v[ch][c] : -INFINITY;
+          }
+          float c0 = v[0][0], c1 = v[0][1], c2m = v[0][2], c3 = v[0][3];
 #pragma unroll
           for (int ch = 0; ch < NCH; ++ch)
 #pragma unroll
-            for (int c = 0; c < 32; ++c)
-              v[ch][c] = (kb + ch * 32 + c <= jmax) ? v[ch][c] : -INFINITY;
+            for (int c = (ch == 0 ? 4 : 0); c < 32; c += 4) {
+              c0 = fmaxf(c0, v[ch][c + 0]);
+              c1 = fmaxf(c1, v[ch][c + 1]);
+              c2m = fmaxf(c2m, v[ch][c + 2]);
+              c3 = fmaxf(c3, v[ch][c + 3]);
+            }
+          const float cmax = fmaxf(fmaxf(c0, c1), fmaxf(c2m, c3));
+          const float mnew = fmaxf(fmaxf(cmax * a.c2, m2), -1e30f);
+          l *= ex2_approx(m2 - mnew);
+          float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+          for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+            for (int c = 0; c < 32; c += 4) {
+              s0 += ex2_approx(fmaf(v[ch][c + 0], a.c2, -mnew));
+              s1 += ex2_approx(fmaf(v[ch][c + 1], a.c2, -mnew));
+              s2 += ex2_approx(fmaf(v[ch][c + 2], a.c2, -mnew));
+              s3 += ex2_approx(fmaf(v[ch][c + 3], a.c2, -mnew));
+            }
+          l += (s0 + s1) + (s2 + s3);
+          m2 = mnew;
         }
-        float c0 = v[0][0], c1 = v[0][1], c2m = v[0][2], c3 = v[0][3];
-#pragma unroll
-        for (int ch = 0; ch < NCH; ++ch)
-#pragma unroll
-          for (int c = (ch == 0 ? 4 : 0); c < 32; c += 4) {
-            c0 = fmaxf(c0, v[ch][c + 0]);
-            c1 = fmaxf(c1, v[ch][c + 1]);
-            c2m = fmaxf(c2m, v[ch][c + 2]);
-            c3 = fmaxf(c3, v[ch][c + 3]);
-          }
-        const float cmax = fmaxf(fmaxf(c0, c1), fmaxf(c2m, c3));
-        const float mnew = fmaxf(fmaxf(cmax * a.c2, m2), -1e30f);
-        l *= ex2_approx(m2 - mnew);
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-        for (int ch = 0; ch < NCH; ++ch)
-#pragma unroll
-          for (int c = 0; c < 32; c += 4) {
-            s0 += ex2_approx(fmaf(v[ch][c + 0], a.c2, -mnew));
-            s1 += ex2_approx(fmaf(v[ch][c + 1], a.c2, -mnew));
-            s2 += ex2_approx(fmaf(v[ch][c + 2], a.c2, -mnew));
-            s3 += ex2_approx(fmaf(v[ch][c + 3], a.c2, -mnew));
-          }
-        l += (s0 + s1) + (s2 + s3);
-        m2 = mnew;
+        // publish this CTA's (max, sum) of the unit: merge replicas and warpgroups first
+        part_s[(wg * 4 + q) * 32 + lane] = make_float2(m2, l);
+        named_bar_sync(1, EPI_THREADS);
+        dead = dead || (*abort_s != 0);
+        const bool good = !dead;
+        if (good && tid < a.ncols) {
+          float M = -INFINITY;
+          for (int w2 = 0; w2 < 2; ++w2)
+            for (int r = 0; r < REPS; ++r) {
+              const int row = r * NPAD + tid;
+              M = fmaxf(M, part_s[(w2 * 4 + (row >> 5)) * 32 + (row & 31)].x);
+            }
+          float S = 0.f;
+          for (int w2 = 0; w2 < 2; ++w2)
+            for (int r = 0; r < REPS; ++r) {
+              const int row = r * NPAD + tid;
+              const float2 p = part_s[(w2 * 4 + (row >> 5)) * 32 + (row & 31)];
+              S += p.y * exp2f(p.x - M);
+            }
+          a.partials[(static_cast<size_t>(it.unit) * a.maxseg + it.slot) * MAX_COLS + tid] =
+              make_float2(M, S);
+          __threadfence();
+        }
+        named_bar_sync(1, EPI_THREADS);
+        if (good && tid == 0) atomicAdd(a.counters + it.unit, 1);
+        return true;
       }
-      part_s[(wg * 4 + q) * 32 + lane] = make_float2(m2, l);
-      named_bar_sync(1, EPI_THREADS);
-      const int tid = threadIdx.x - 64;
-      const bool aborted = (*abort_s != 0);
-      if (!aborted && tid < a.ncols) {
-        // merge the replicas and the two warpgroups of this CTA, fixed order
-        const int reps = 128 / a.npad;
-        float M = -INFINITY;
-        for (int w2 = 0; w2 < 2; ++w2)
-          for (int r = 0; r < reps; ++r) {
-            const int row = r * a.npad + tid;
-            M = fmaxf(M, part_s[(w2 * 4 + (row >> 5)) * 32 + (row & 31)].x);
+      // ------------------------------------------------------------ votes
+      // every partial of the unit must have been published (bounded wait), then the
+      // log2-sum-exp of each window row is merged from them in slot order
+      named_bar_sync(1, EPI_THREADS);  // both warpgroups are done with the previous lse_s
+      if (warp == 2 && !dead) {
+        int seen = 0;
+        if (lane == 0) {
+          seen = ld_acquire(a.counters + it.unit);
+          if (seen < it.nseg) {
+            const unsigned long long t0 = globaltimer_ns();
+            for (;;) {
+              seen = ld_acquire(a.counters + it.unit);
+              if (seen >= it.nseg || *abort_s != 0) break;
+              if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort_s = WAIT_UNIT_STATS; break; }
+              __nanosleep(200);
+            }
           }
-        float S = 0.f;
-        for (int w2 = 0; w2 < 2; ++w2)
-          for (int r = 0; r < reps; ++r) {
-            const int row = r * a.npad + tid;
-            const float2 p = part_s[(w2 * 4 + (row >> 5)) * 32 + (row & 31)];
+        }
+      }
+      named_bar_sync(1, EPI_THREADS);
+      dead = dead || (*abort_s != 0);
+      if (tid < MAX_COLS) {
+        float val = 0.f;
+        if (tid < a.ncols && !dead) {
+          const float2* pp = a.partials + static_cast<size_t>(it.unit) * a.maxseg * MAX_COLS + tid;
+          float M = -INFINITY;
+          for (int c = 0; c < it.nseg; ++c) M = fmaxf(M, __ldcg(pp + c * MAX_COLS).x);
+          float S = 0.f;
+          for (int c = 0; c < it.nseg; ++c) {
+            const float2 p = __ldcg(pp + c * MAX_COLS);
             S += p.y * exp2f(p.x - M);
           }
-        a.partials[(static_cast<size_t>(u) * a.chunks + chunk) * MAX_COLS + tid] = make_float2(M, S);
-      }
-      __threadfence();
-      named_bar_sync(1, EPI_THREADS);
-      if (tid == 0 && !aborted) {
-        const int old = atomicAdd(a.counters + u, 1);
-        *last_s = (old == a.chunks - 1) ? 1 : 0;
-      }
-      named_bar_sync(1, EPI_THREADS);
-      if (*last_s != 0 && tid < a.ncols) {
-        // this CTA finished last for the unit: every partial is visible now
-        __threadfence();
-        const float2* pp = a.partials + static_cast<size_t>(u) * a.chunks * MAX_COLS + tid;
-        float M = -INFINITY;
-        for (int c = 0; c < a.chunks; ++c) M = fmaxf(M, __ldcg(pp + c * MAX_COLS).x);
-        float S = 0.f;
-        for (int c = 0; c < a.chunks; ++c) {
-          const float2 p = __ldcg(pp + c * MAX_COLS);
-          S += p.y * exp2f(p.x - M);
+          val = -(M + log2f(S));
         }
-        a.lse2[static_cast<size_t>(u) * MAX_COLS + tid] = M + log2f(S);
+        lse_s[tid] = val;
       }
-    } else {
-      // ---------------------------------------------------------- votes
-      const bool w16 = (a.W & 15) == 0;
-      const int gpw = a.W >> 4;  // 16-column groups per head (when W is a multiple of 16)
-      for (int it = wg; it < nt; it += 2) {
-        const int buf = it & (NBUF - 1);
-        const uint32_t ub = (it / NBUF) & 1;
-        if (!mbar_wait_warp(bar_tf(buf), ub, abort_s, WAIT_EPI_TMEM_FULL)) break;
+      named_bar_sync(1, EPI_THREADS);
+      for (int k = 0; k < nt; ++k, ++git) {
+        if ((git & 1) != wg || dead) continue;
+        const int buf = git & (NBUF - 1);
+        const uint32_t ub = (git / NBUF) & 1;
+        if (!mbar_wait_warp(bar_tf(buf), ub, abort_s, WAIT_EPI_TMEM_FULL)) {
+          dead = true;
+          continue;
+        }
         tc_fence_after();
-        const int j = tile_of(it) * TILE_KEYS + 32 * q + lane;
+        const int j = tile_of(it, k) * TILE_KEYS + 32 * q + lane;
         const uint32_t taddr = tmem_base + lane_sel + buf * 128;
         // this key's logits against every window row of the unit
         float v[NCH][32];
@@ -395,7 +525,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             }
         }
       }
-    }
+      return true;
+    });
   }
 
   tc_fence_before();
@@ -440,34 +571,40 @@ bool encode_map(CUtensorMap* m, const void* base, int rank, const cuuint64_t* di
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SM_COUNT_HINT;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
+      n = SM_COUNT_HINT;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
 template <int D, int NCH>
-cudaError_t run_passes(const CUtensorMap& tmK, const CUtensorMap& tmQ, ScoreArgs a,
-                       const ScorePlan& p, cudaStream_t stream, int* launches) {
+cudaError_t run_scores(const CUtensorMap& tmK, const CUtensorMap& tmQ, const ScoreArgs& a,
+                       int grid, cudaStream_t stream, int* launches) {
   static bool attr_done = false;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(score_kernel<D, false, NCH>,
+    cudaError_t e = cudaFuncSetAttribute(score_kernel<D, NCH>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          Smem<D>::DYN_BYTES);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(score_kernel<D, true, NCH>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::DYN_BYTES);
-    if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  for (int u0 = 0; u0 < p.units; u0 += p.units_per_wave) {
-    const int nu = (p.units - u0 < p.units_per_wave) ? (p.units - u0) : p.units_per_wave;
-    a.unit0 = u0;
-    a.tiles = p.tiles_stats;
-    a.chunks = p.chunks_stats;
-    score_kernel<D, false, NCH><<<dim3(p.chunks_stats, nu), THREADS, Smem<D>::DYN_BYTES, stream>>>(
-        tmK, tmQ, a);
-    a.tiles = p.tiles_vote;
-    a.chunks = p.chunks_vote;
-    score_kernel<D, true, NCH><<<dim3(p.chunks_vote, nu), THREADS, Smem<D>::DYN_BYTES, stream>>>(
-        tmK, tmQ, a);
-    *launches += 2;
-  }
-  return cudaGetLastError();
+  void* params[3] = {const_cast<CUtensorMap*>(&tmK), const_cast<CUtensorMap*>(&tmQ),
+                     const_cast<ScoreArgs*>(&a)};
+  // cooperative launch: every CTA is resident, so a CTA that waits for another CTA's
+  // partial statistics cannot keep that CTA off the machine
+  cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(score_kernel<D, NCH>),
+                                              dim3(grid), dim3(THREADS), params,
+                                              Smem<D>::DYN_BYTES, stream);
+  if (e != cudaSuccess) return e;
+  *launches += 1;
+  return cudaSuccess;
 }
 
 }  // namespace
@@ -489,31 +626,37 @@ bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* pla
   const int n = L - W;
   p.tiles_stats = (L + TILE_KEYS - 1) / TILE_KEYS;
   p.tiles_vote = (n + TILE_KEYS - 1) / TILE_KEYS;
-  // A wave is the set of units whose keys are swept twice back to back; it is sized so
-  // that the second sweep finds the keys in L2 (64 MiB of K per wave).
+  // A wave is a set of units whose keys are swept twice; with the pipelined schedule two
+  // waves are live in L2 at a time, so a wave holds about 32 MiB of keys.  Units too big
+  // for that take the sequential schedule, one unit per wave.
   const long long kbytes = static_cast<long long>(L) * d * 2;
-  long long kv_per_wave = (64ll << 20) / kbytes;
+  long long kv_per_wave = (32ll << 20) / kbytes;
+  p.pipelined = kv_per_wave >= 1 ? 1 : 0;
   if (kv_per_wave < 1) kv_per_wave = 1;
-  if (kv_per_wave > 4096) kv_per_wave = 4096;
+  if (kv_per_wave > 1024) kv_per_wave = 1024;
   long long upw = kv_per_wave * p.sub_per_kv;
   if (upw > units) upw = units;
   p.units_per_wave = static_cast<int>(upw);
-  auto chunks_for = [&](int tiles) {
-    int c = SM_COUNT_HINT / p.units_per_wave;
-    if (c < 1) c = 1;
-    if (c > tiles) c = tiles;
-    if (c < 1) c = 1;
-    return c;
+  p.nwaves = (p.units + p.units_per_wave - 1) / p.units_per_wave;
+  // partial slots per unit: a unit of T1 tiles is shared by at most ceil(T1 / q) + 1 CTAs
+  // when every CTA gets at least q = floor(TT / G) tiles of the wave (G up to MAX_GRID)
+  auto segs = [&](int nu) {
+    const long long TT = static_cast<long long>(nu) * p.tiles_stats;
+    const long long q = TT / MAX_GRID;
+    long long s = q >= 1 ? (p.tiles_stats + q - 1) / q + 1 : p.tiles_stats;
+    if (s > MAX_GRID) s = MAX_GRID;
+    return static_cast<int>(s);
   };
-  p.chunks_stats = chunks_for(p.tiles_stats);
-  p.chunks_vote = chunks_for(p.tiles_vote);
+  const int last_nu = p.units - (p.nwaves - 1) * p.units_per_wave;
+  p.maxseg = segs(p.units_per_wave);
+  if (segs(last_nu) > p.maxseg) p.maxseg = segs(last_nu);
   *plan = p;
   return true;
 }
 
 cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv, int L,
                                  int d, int W, const ScorePlan& plan, float* vote, int* status,
-                                 int* counters, float2* partials, float* lse2, cudaStream_t stream,
+                                 int* counters, float2* partials, cudaStream_t stream,
                                  int* launches) {
   CUtensorMap tmK, tmQ;
   {
@@ -540,24 +683,29 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq
   a.npad = plan.npad;
   a.sub_per_kv = plan.sub_per_kv;
   a.g = plan.g;
-  a.tiles = 0;
-  a.chunks = 0;
-  a.unit0 = 0;
+  a.units = plan.units;
+  a.upw = plan.units_per_wave;
+  a.nwaves = plan.nwaves;
+  a.T1 = plan.tiles_stats;
+  a.T2 = plan.tiles_vote;
+  a.maxseg = plan.maxseg;
+  a.pipelined = plan.pipelined;
   a.c2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
   a.partials = partials;
-  a.lse2 = lse2;
   a.counters = counters;
   a.status = status;
   a.vote = vote;
+  int grid = sm_count();
+  if (grid > MAX_GRID) grid = MAX_GRID;
   const int nch = plan.npad >> 5;
   if (d == 64) {
-    if (nch == 1) return run_passes<64, 1>(tmK, tmQ, a, plan, stream, launches);
-    if (nch == 2) return run_passes<64, 2>(tmK, tmQ, a, plan, stream, launches);
-    return run_passes<64, 4>(tmK, tmQ, a, plan, stream, launches);
+    if (nch == 1) return run_scores<64, 1>(tmK, tmQ, a, grid, stream, launches);
+    if (nch == 2) return run_scores<64, 2>(tmK, tmQ, a, grid, stream, launches);
+    return run_scores<64, 4>(tmK, tmQ, a, grid, stream, launches);
   }
-  if (nch == 1) return run_passes<128, 1>(tmK, tmQ, a, plan, stream, launches);
-  if (nch == 2) return run_passes<128, 2>(tmK, tmQ, a, plan, stream, launches);
-  return run_passes<128, 4>(tmK, tmQ, a, plan, stream, launches);
+  if (nch == 1) return run_scores<128, 1>(tmK, tmQ, a, grid, stream, launches);
+  if (nch == 2) return run_scores<128, 2>(tmK, tmQ, a, grid, stream, launches);
+  return run_scores<128, 4>(tmK, tmQ, a, grid, stream, launches);
 }
 
 }  // namespace snapkv
