@@ -22,6 +22,10 @@ enum WaitCode {
   WAIT_Q_FULL = 5,
   WAIT_DRAIN = 6,
   WAIT_UNIT_STATS = 7,
+  WAIT_PART_EMPTY = 8,
+  WAIT_PART_FULL = 9,
+  WAIT_LSE_FULL = 10,
+  WAIT_LSE_EMPTY = 11,
 };
 
 // How the scoring passes split the work.  A "unit" is one (batch, KV head, head

@@ -25,7 +25,9 @@
 // Warp roles: warp 0 issues TMA loads (K tiles into a ring of stages, Q per work item
 // into two buffers), warp 1 issues tcgen05.mma into four TMEM accumulator buffers, warps
 // 2-9 (two warpgroups, alternating tiles) read the accumulators back with tcgen05.ld and
-// do the fp32 softmax arithmetic.
+// do the fp32 softmax arithmetic, warp 10 is the book-keeper: it merges and publishes the
+// partial statistics the softmax warps leave in shared memory, and prepares the merged
+// log-sum-exp of the next vote item while the softmax warps are still busy.
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <math.h>
@@ -42,8 +44,10 @@ constexpr int STAGES = 4;
 constexpr int NBUF = 4;               // TMEM accumulator buffers of 128 columns
 constexpr int TMEM_COLS = 512;
 constexpr int SUBTILE_BYTES = 128 * 128;  // 128 rows x 64 bf16, 128-byte swizzled
-constexpr int THREADS = 320;          // producer warp, MMA warp, 8 epilogue warps
-constexpr int EPI_THREADS = 256;
+constexpr int THREADS = 352;          // producer, MMA, 8 softmax warps, book-keeper
+constexpr int EPI_WARPS = 8;
+constexpr int NPB = 4;                // buffers for partial statistics (book-keeper queue)
+constexpr int NLB = 8;                // buffers for merged log-sum-exp rows
 
 struct ScoreArgs {
   int L, n, W;
@@ -68,12 +72,14 @@ struct Smem {
   static constexpr int OFF_Q = 0;                            // two Q buffers
   static constexpr int OFF_K = 2 * Q_BYTES;
   static constexpr int OFF_BAR = OFF_K + STAGES * STAGE_BYTES;
-  // barriers: full[STAGES], empty[STAGES], tf[NBUF], te[NBUF], qfull[2], qempty[2], drain
-  static constexpr int NBAR = 2 * STAGES + 2 * NBUF + 5;
-  static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;       // tmem ptr, abort
-  static constexpr int OFF_PART = OFF_MISC + 24;            // float2 [8][32]
-  static constexpr int OFF_LSE = OFF_PART + 8 * 32 * 8;     // float [128]
-  static constexpr int TOTAL = OFF_LSE + 128 * 4;
+  // barriers: full[STAGES], empty[STAGES], tf[NBUF], te[NBUF], qfull[2], qempty[2], drain,
+  // pfull[NPB], pempty[NPB] (partial statistics), lfull[NLB], lempty[NLB] (log-sum-exp)
+  static constexpr int NBAR = 2 * STAGES + 2 * NBUF + 5 + 2 * NPB + 2 * NLB;
+  static constexpr int OFF_MISC = OFF_BAR + ((NBAR * 8 + 15) & ~15);  // tmem ptr, abort
+  static constexpr int OFF_PART = OFF_MISC + 16;              // float2 [NPB][8][32]
+  static constexpr int OFF_LSE = OFF_PART + NPB * 8 * 32 * 8; // float [NLB][128]
+  static constexpr int TOTAL = OFF_LSE + NLB * 128 * 4;
+  static_assert(OFF_PART % 16 == 0 && OFF_LSE % 16 == 0, "float4 reads of the lse buffers");
   static constexpr int DYN_BYTES = TOTAL + 1024;            // slack for 1024-byte alignment
 };
 
@@ -83,6 +89,24 @@ __device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity) {
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) return false;
+  }
+}
+
+// Warp-wide wait for a warp that is off the critical path: backs off between polls so
+// that it does not take issue slots from the softmax warps of its scheduler.
+__device__ __forceinline__ bool mbar_wait_warp_relaxed(uint32_t bar, uint32_t parity,
+                                                       volatile int* abort_flag, int code) {
+  if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  for (;;) {
+    __nanosleep(250);
+    if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+    int stop = 0;
+    if ((threadIdx.x & 31) == 0) {
+      if (*abort_flag != 0) stop = 1;
+      else if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = code; stop = 1; }
+    }
+    if (__shfl_sync(0xffffffffu, stop, 0)) return false;
   }
 }
 
@@ -107,11 +131,12 @@ __device__ __forceinline__ int cta_of_tile(long long x, long long TT, int G) {
 // Calls f(item) for every work item of this CTA in schedule order; stops when f
 // returns false.  All three warp roles walk the same list.
 template <typename F>
-__device__ __forceinline__ void for_each_item(const ScoreArgs& a, int cta, int G, F&& f) {
+__device__ __forceinline__ void for_each_item(const ScoreArgs& a, int cta, int G, bool pipelined,
+                                              F&& f) {
   const int nph = 2 * a.nwaves;
   for (int p = 0; p < nph; ++p) {
     int w, vote;
-    if (a.pipelined) {
+    if (pipelined) {
       if (p == 0) { w = 0; vote = 0; }
       else if (p == nph - 1) { w = a.nwaves - 1; vote = 1; }
       else if (p & 1) { w = (p + 1) >> 1; vote = 0; }
@@ -173,6 +198,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   auto bar_qf = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 * NBUF + b); };
   auto bar_qe = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 * NBUF + 2 + b); };
   const uint32_t bar_drain = bar0 + 8u * (2 * STAGES + 2 * NBUF + 4);
+  constexpr int BAR_P = 2 * STAGES + 2 * NBUF + 5;
+  auto bar_pf = [&](int b) { return bar0 + 8u * (BAR_P + b); };
+  auto bar_pe = [&](int b) { return bar0 + 8u * (BAR_P + NPB + b); };
+  auto bar_lf = [&](int b) { return bar0 + 8u * (BAR_P + 2 * NPB + b); };
+  auto bar_le = [&](int b) { return bar0 + 8u * (BAR_P + 2 * NPB + NLB + b); };
   volatile uint32_t* tmem_ptr_s = reinterpret_cast<volatile uint32_t*>(smem + SM::OFF_MISC);
   volatile int* abort_s = reinterpret_cast<volatile int*>(smem + SM::OFF_MISC + 4);
   float2* part_s = reinterpret_cast<float2*>(smem + SM::OFF_PART);
@@ -195,6 +225,14 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar_qf(b), 1);
       mbar_init(bar_qe(b), 1);
+    }
+    for (int b = 0; b < NPB; ++b) {
+      mbar_init(bar_pf(b), EPI_WARPS);
+      mbar_init(bar_pe(b), 1);
+    }
+    for (int b = 0; b < NLB; ++b) {
+      mbar_init(bar_lf(b), 1);
+      mbar_init(bar_le(b), EPI_WARPS);
     }
     mbar_init(bar_drain, 1);
     *abort_s = 0;
@@ -226,7 +264,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       tma_prefetch_desc(&tmQ);
       int git = 0;      // tiles issued so far (ring position)
       int nitem = 0;    // items started so far (Q buffer position)
-      for_each_item(a, cta, G, [&](const Item& it) {
+      for_each_item(a, cta, G, a.pipelined != 0, [&](const Item& it) {
         int ukv;
         const int qrow0 = first_head(it.unit, &ukv) * a.W;
         const int qb = nitem & 1;
@@ -276,7 +314,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       const uint32_t idesc_s = umma_idesc_bf16(128, 128);
       const uint32_t idesc_v = umma_idesc_bf16(128, NPAD);
       int git = 0, nitem = 0;
-      for_each_item(a, cta, G, [&](const Item& it) {
+      for_each_item(a, cta, G, a.pipelined != 0, [&](const Item& it) {
         const int qb = nitem & 1;
         if (!mbar_wait_thread(bar_qf(qb), (nitem >> 1) & 1, abort_s, WAIT_Q_FULL)) return false;
         ++nitem;
@@ -312,24 +350,19 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         mbar_wait_drain(bar_drain, 0);
       }
     }
-  } else {
+  } else if (warp < 2 + EPI_WARPS) {
     // ------------------------------------------------------------ softmax warps
     const int wg = (warp - 2) >> 2;
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     const uint32_t lane_sel = static_cast<uint32_t>(32 * q) << 16;
-    const int tid = threadIdx.x - 64;
     const int rrow = 32 * q + lane;  // TMEM lane
     const int rep = rrow / NPAD;
     const int qcol = rrow - rep * NPAD;
     const int jmax = min(a.L - 1, a.n + (qcol % a.W));  // last key window row qcol % W sees
     const bool w16 = (a.W & 15) == 0;
     const int gpw = a.W >> 4;  // 16-column groups per head (when W is a multiple of 16)
-    int git = 0;
-    // Once a wait has given up (here or in another role) this warp stops touching TMEM
-    // and barriers of the pipeline but still walks every item, so that all eight warps
-    // keep meeting at the named barriers and reach the end of the kernel together.
-    bool dead = false;
-    for_each_item(a, cta, G, [&](const Item& it) {
+    int git = 0, nstat = 0, nvote = 0;
+    for_each_item(a, cta, G, a.pipelined != 0, [&](const Item& it) {
       const int nt = it.t1 - it.t0;
       int ukv;
       const int hq0 = first_head(it.unit, &ukv);
@@ -338,13 +371,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         float m2 = -INFINITY;  // running max, log2 domain
         float l = 0.f;         // running sum of exp2(x - m2)
         for (int k = 0; k < nt; ++k, ++git) {
-          if ((git & 1) != wg || dead) continue;
+          if ((git & 1) != wg) continue;
           const int buf = git & (NBUF - 1);
           const uint32_t ub = (git / NBUF) & 1;
-          if (!mbar_wait_warp(bar_tf(buf), ub, abort_s, WAIT_EPI_TMEM_FULL)) {
-            dead = true;
-            continue;
-          }
+          if (!mbar_wait_warp(bar_tf(buf), ub, abort_s, WAIT_EPI_TMEM_FULL)) return false;
           tc_fence_after();
           const int key0 = tile_of(it, k) * TILE_KEYS;
           // the whole slice of this thread's row: NPAD key columns
@@ -391,78 +421,25 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           l += (s0 + s1) + (s2 + s3);
           m2 = mnew;
         }
-        // publish this CTA's (max, sum) of the unit: merge replicas and warpgroups first
-        part_s[(wg * 4 + q) * 32 + lane] = make_float2(m2, l);
-        named_bar_sync(1, EPI_THREADS);
-        dead = dead || (*abort_s != 0);
-        const bool good = !dead;
-        if (good && tid < a.ncols) {
-          float M = -INFINITY;
-          for (int w2 = 0; w2 < 2; ++w2)
-            for (int r = 0; r < REPS; ++r) {
-              const int row = r * NPAD + tid;
-              M = fmaxf(M, part_s[(w2 * 4 + (row >> 5)) * 32 + (row & 31)].x);
-            }
-          float S = 0.f;
-          for (int w2 = 0; w2 < 2; ++w2)
-            for (int r = 0; r < REPS; ++r) {
-              const int row = r * NPAD + tid;
-              const float2 p = part_s[(w2 * 4 + (row >> 5)) * 32 + (row & 31)];
-              S += p.y * exp2f(p.x - M);
-            }
-          a.partials[(static_cast<size_t>(it.unit) * a.maxseg + it.slot) * MAX_COLS + tid] =
-              make_float2(M, S);
-          __threadfence();
-        }
-        named_bar_sync(1, EPI_THREADS);
-        if (good && tid == 0) atomicAdd(a.counters + it.unit, 1);
+        // leave this warp's (max, sum) per TMEM lane for the book-keeper
+        const int pb = nstat % NPB;
+        if (!mbar_wait_warp(bar_pe(pb), ((nstat / NPB) & 1) ^ 1, abort_s, WAIT_PART_EMPTY))
+          return false;
+        part_s[(pb * 8 + wg * 4 + q) * 32 + lane] = make_float2(m2, l);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_pf(pb));
+        ++nstat;
         return true;
       }
       // ------------------------------------------------------------ votes
-      // every partial of the unit must have been published (bounded wait), then the
-      // log2-sum-exp of each window row is merged from them in slot order
-      named_bar_sync(1, EPI_THREADS);  // both warpgroups are done with the previous lse_s
-      if (warp == 2 && !dead) {
-        int seen = 0;
-        if (lane == 0) {
-          seen = ld_acquire(a.counters + it.unit);
-          if (seen < it.nseg) {
-            const unsigned long long t0 = globaltimer_ns();
-            for (;;) {
-              seen = ld_acquire(a.counters + it.unit);
-              if (seen >= it.nseg || *abort_s != 0) break;
-              if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort_s = WAIT_UNIT_STATS; break; }
-              __nanosleep(200);
-            }
-          }
-        }
-      }
-      named_bar_sync(1, EPI_THREADS);
-      dead = dead || (*abort_s != 0);
-      if (tid < MAX_COLS) {
-        float val = 0.f;
-        if (tid < a.ncols && !dead) {
-          const float2* pp = a.partials + static_cast<size_t>(it.unit) * a.maxseg * MAX_COLS + tid;
-          float M = -INFINITY;
-          for (int c = 0; c < it.nseg; ++c) M = fmaxf(M, __ldcg(pp + c * MAX_COLS).x);
-          float S = 0.f;
-          for (int c = 0; c < it.nseg; ++c) {
-            const float2 p = __ldcg(pp + c * MAX_COLS);
-            S += p.y * exp2f(p.x - M);
-          }
-          val = -(M + log2f(S));
-        }
-        lse_s[tid] = val;
-      }
-      named_bar_sync(1, EPI_THREADS);
+      const int lb = nvote % NLB;
+      if (!mbar_wait_warp(bar_lf(lb), (nvote / NLB) & 1, abort_s, WAIT_LSE_FULL)) return false;
+      const float* lse_b = lse_s + lb * MAX_COLS;
       for (int k = 0; k < nt; ++k, ++git) {
-        if ((git & 1) != wg || dead) continue;
+        if ((git & 1) != wg) continue;
         const int buf = git & (NBUF - 1);
         const uint32_t ub = (git / NBUF) & 1;
-        if (!mbar_wait_warp(bar_tf(buf), ub, abort_s, WAIT_EPI_TMEM_FULL)) {
-          dead = true;
-          continue;
-        }
+        if (!mbar_wait_warp(bar_tf(buf), ub, abort_s, WAIT_EPI_TMEM_FULL)) return false;
         tc_fence_after();
         const int j = tile_of(it, k) * TILE_KEYS + 32 * q + lane;
         const uint32_t taddr = tmem_base + lane_sel + buf * 128;
@@ -481,7 +458,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           for (int ch = 0; ch < NCH; ++ch)
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
-              const float4* nl = reinterpret_cast<const float4*>(lse_s + ch * 32 + hf * 16);
+              const float4* nl = reinterpret_cast<const float4*>(lse_b + ch * 32 + hf * 16);
               float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
               for (int t4 = 0; t4 < 4; ++t4) {
@@ -514,7 +491,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             for (int c = 0; c < 32; ++c) {
               const int col = ch * 32 + c;
               if (col < a.ncols) {
-                acc += ex2_approx(fmaf(v[ch][c], a.c2, lse_s[col]));
+                acc += ex2_approx(fmaf(v[ch][c], a.c2, lse_b[col]));
                 if (--left == 0) {
                   if (j < a.n) a.vote[static_cast<size_t>(hq0 + hl) * a.n + j] = acc;
                   acc = 0.f;
@@ -525,6 +502,87 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             }
         }
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_le(lb));  // this warp is done reading lse_s[lb]
+      ++nvote;
+      return true;
+    });
+  } else {
+    // ------------------------------------------------------------ book-keeper warp
+    // It walks the waves in the order S(0) V(0) S(1) V(1) ...: the same statistics items
+    // and the same vote items as the other roles, each kind in the same relative order,
+    // but the log-sum-exp of wave w is prepared right after wave w's statistics are
+    // published, a whole phase before the softmax warps ask for it.
+    int nstat = 0, nvote = 0;
+    for_each_item(a, cta, G, /*pipelined=*/false, [&](const Item& it) {
+      if (!it.vote) {
+        // merge the replicas and the two warpgroups (fixed order), publish, count
+        const int pb = nstat % NPB;
+        if (!mbar_wait_warp_relaxed(bar_pf(pb), (nstat / NPB) & 1, abort_s, WAIT_PART_FULL))
+          return false;
+        const float2* ps = part_s + pb * 8 * 32;
+        for (int c = lane; c < a.ncols; c += 32) {
+          float M = -INFINITY;
+          for (int w2 = 0; w2 < 2; ++w2)
+            for (int r = 0; r < REPS; ++r) {
+              const int row = r * NPAD + c;
+              M = fmaxf(M, ps[(w2 * 4 + (row >> 5)) * 32 + (row & 31)].x);
+            }
+          float S = 0.f;
+          for (int w2 = 0; w2 < 2; ++w2)
+            for (int r = 0; r < REPS; ++r) {
+              const int row = r * NPAD + c;
+              const float2 p = ps[(w2 * 4 + (row >> 5)) * 32 + (row & 31)];
+              S += p.y * exp2f(p.x - M);
+            }
+          a.partials[(static_cast<size_t>(it.unit) * a.maxseg + it.slot) * MAX_COLS + c] =
+              make_float2(M, S);
+        }
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) {
+          atomicAdd(a.counters + it.unit, 1);
+          mbar_arrive(bar_pe(pb));
+        }
+        ++nstat;
+        return true;
+      }
+      // the merged log2-sum-exp of the unit's window rows, as soon as every partial of the
+      // unit has been published (bounded wait) and the softmax warps are done with the
+      // buffer it goes into
+      const int lb = nvote % NLB;
+      if (!mbar_wait_warp_relaxed(bar_le(lb), ((nvote / NLB) & 1) ^ 1, abort_s, WAIT_LSE_EMPTY))
+        return false;
+      int stop = 0;
+      if (lane == 0 && ld_acquire(a.counters + it.unit) < it.nseg) {
+        const unsigned long long t0 = globaltimer_ns();
+        for (;;) {
+          if (ld_acquire(a.counters + it.unit) >= it.nseg) break;
+          if (*abort_s != 0) { stop = 1; break; }
+          if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort_s = WAIT_UNIT_STATS; stop = 1; break; }
+          __nanosleep(100);
+        }
+      }
+      if (__shfl_sync(0xffffffffu, stop, 0)) return false;
+      (void)ld_acquire(a.counters + it.unit);  // every lane orders its reads after the count
+      for (int c = lane; c < MAX_COLS; c += 32) {
+        float val = 0.f;
+        if (c < a.ncols) {
+          const float2* pp = a.partials + static_cast<size_t>(it.unit) * a.maxseg * MAX_COLS + c;
+          float M = -INFINITY;
+          for (int sgi = 0; sgi < it.nseg; ++sgi) M = fmaxf(M, __ldcg(pp + sgi * MAX_COLS).x);
+          float S = 0.f;
+          for (int sgi = 0; sgi < it.nseg; ++sgi) {
+            const float2 p = __ldcg(pp + sgi * MAX_COLS);
+            S += p.y * exp2f(p.x - M);
+          }
+          val = -(M + log2f(S));
+        }
+        lse_s[lb * MAX_COLS + c] = val;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_lf(lb));
+      ++nvote;
       return true;
     });
   }
@@ -633,8 +691,11 @@ bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* pla
   long long kv_per_wave = (32ll << 20) / kbytes;
   p.pipelined = kv_per_wave >= 1 ? 1 : 0;
   if (kv_per_wave < 1) kv_per_wave = 1;
-  if (kv_per_wave > 1024) kv_per_wave = 1024;
   long long upw = kv_per_wave * p.sub_per_kv;
+  // at most 128 units per wave: a CTA's share of a phase then spans few units, which
+  // bounds the work items per phase (the book-keeper's buffers are sized for that)
+  if (upw > 128) upw = 128 / p.sub_per_kv * p.sub_per_kv;
+  if (upw < p.sub_per_kv) upw = p.sub_per_kv;
   if (upw > units) upw = units;
   p.units_per_wave = static_cast<int>(upw);
   p.nwaves = (p.units + p.units_per_wave - 1) / p.units_per_wave;
