@@ -46,7 +46,7 @@ struct ScorePlan {
 };
 
 struct WorkspaceLayout {
-  size_t off_status, off_counters, off_partials, off_vote, off_pooled, total;
+  size_t off_status, off_counters, off_partials, off_lse, off_vote, off_pooled, total;
 };
 
 bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* plan);
@@ -57,7 +57,7 @@ bool select_needs_scratch(int n);
 // Enqueue both scoring passes.  `vote` is fp32 [B*Hq, n].
 cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv, int L,
                                  int d, int W, const ScorePlan& plan, float* vote, int* status,
-                                 int* counters, float2* partials, cudaStream_t stream,
+                                 int* counters, float2* partials, float* lse2, cudaStream_t stream,
                                  int* launches);
 
 // Pool + top-k over `rows` rows of fp32 votes.  `pooled_scratch` (fp32 [rows, n]) is

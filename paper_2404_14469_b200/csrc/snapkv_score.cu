@@ -59,7 +59,8 @@ struct ScoreArgs {
   int pipelined;            // phase order S0 S1 V0 S2 V1 ... (else S0 V0 S1 V1 ...)
   float c2;                 // log2(e) / sqrt(d)
   float2* partials;         // [units][maxseg][MAX_COLS] (max, sum) in the log2 domain
-  int* counters;            // [units] published partials
+  float* lse2;              // [units][MAX_COLS] minus the merged log2-sum-exp per window row
+  int* counters;            // [units] published partials (+1 once lse2 is written)
   int* status;
   float* vote;
 };
@@ -540,24 +541,69 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         }
         __threadfence();
         __syncwarp();
+        int last = 0;
         if (lane == 0) {
-          atomicAdd(a.counters + it.unit, 1);
+          last = (atomicAdd(a.counters + it.unit, 1) == it.nseg - 1) ? 1 : 0;
           mbar_arrive(bar_pe(pb));
+        }
+        if (__shfl_sync(0xffffffffu, last, 0)) {
+          // this was the unit's last partial: fold all of them, in slot order, into one
+          // -log2-sum-exp per window row, then raise the count once more to say so.
+          // Each lane owns four adjacent window rows; loads go eight segments at a time.
+          (void)ld_acquire(a.counters + it.unit);
+          const int c4 = lane * 4;
+          if (c4 < a.ncols) {
+            const float4* pp = reinterpret_cast<const float4*>(
+                a.partials + static_cast<size_t>(it.unit) * a.maxseg * MAX_COLS + c4);
+            float M[4], S[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) { M[t] = -INFINITY; S[t] = 0.f; }
+            for (int s0 = 0; s0 < it.nseg; s0 += 8) {
+              float4 x[8][2];
+#pragma unroll
+              for (int uu = 0; uu < 8; ++uu)
+                if (s0 + uu < it.nseg) {
+                  x[uu][0] = __ldcg(pp + static_cast<size_t>(s0 + uu) * (MAX_COLS / 2));
+                  x[uu][1] = __ldcg(pp + static_cast<size_t>(s0 + uu) * (MAX_COLS / 2) + 1);
+                }
+#pragma unroll
+              for (int uu = 0; uu < 8; ++uu)
+                if (s0 + uu < it.nseg) {
+                  const float m[4] = {x[uu][0].x, x[uu][0].z, x[uu][1].x, x[uu][1].z};
+                  const float sv[4] = {x[uu][0].y, x[uu][0].w, x[uu][1].y, x[uu][1].w};
+#pragma unroll
+                  for (int t = 0; t < 4; ++t) {
+                    const float Mn = fmaxf(M[t], m[t]);
+                    S[t] = S[t] * exp2f(M[t] - Mn) + sv[t] * exp2f(m[t] - Mn);
+                    M[t] = Mn;
+                  }
+                }
+            }
+            float4 out;
+            out.x = -(M[0] + log2f(S[0]));
+            out.y = -(M[1] + log2f(S[1]));
+            out.z = -(M[2] + log2f(S[2]));
+            out.w = -(M[3] + log2f(S[3]));
+            *reinterpret_cast<float4*>(a.lse2 + static_cast<size_t>(it.unit) * MAX_COLS + c4) = out;
+          }
+          __threadfence();
+          __syncwarp();
+          if (lane == 0) atomicAdd(a.counters + it.unit, 1);
         }
         ++nstat;
         return true;
       }
-      // the merged log2-sum-exp of the unit's window rows, as soon as every partial of the
-      // unit has been published (bounded wait) and the softmax warps are done with the
-      // buffer it goes into
+      // the merged -log2-sum-exp of the unit's window rows goes into a shared-memory
+      // buffer as soon as the unit's count says it is ready (bounded wait) and the softmax
+      // warps are done with that buffer
       const int lb = nvote % NLB;
       if (!mbar_wait_warp_relaxed(bar_le(lb), ((nvote / NLB) & 1) ^ 1, abort_s, WAIT_LSE_EMPTY))
         return false;
       int stop = 0;
-      if (lane == 0 && ld_acquire(a.counters + it.unit) < it.nseg) {
+      if (lane == 0 && ld_acquire(a.counters + it.unit) <= it.nseg) {
         const unsigned long long t0 = globaltimer_ns();
         for (;;) {
-          if (ld_acquire(a.counters + it.unit) >= it.nseg) break;
+          if (ld_acquire(a.counters + it.unit) > it.nseg) break;
           if (*abort_s != 0) { stop = 1; break; }
           if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort_s = WAIT_UNIT_STATS; stop = 1; break; }
           __nanosleep(100);
@@ -565,20 +611,12 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       }
       if (__shfl_sync(0xffffffffu, stop, 0)) return false;
       (void)ld_acquire(a.counters + it.unit);  // every lane orders its reads after the count
-      for (int c = lane; c < MAX_COLS; c += 32) {
-        float val = 0.f;
-        if (c < a.ncols) {
-          const float2* pp = a.partials + static_cast<size_t>(it.unit) * a.maxseg * MAX_COLS + c;
-          float M = -INFINITY;
-          for (int sgi = 0; sgi < it.nseg; ++sgi) M = fmaxf(M, __ldcg(pp + sgi * MAX_COLS).x);
-          float S = 0.f;
-          for (int sgi = 0; sgi < it.nseg; ++sgi) {
-            const float2 p = __ldcg(pp + sgi * MAX_COLS);
-            S += p.y * exp2f(p.x - M);
-          }
-          val = -(M + log2f(S));
-        }
-        lse_s[lb * MAX_COLS + c] = val;
+      {
+        const int c4 = lane * 4;
+        float4 val = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c4 < a.ncols)
+          val = __ldcg(reinterpret_cast<const float4*>(a.lse2 + static_cast<size_t>(it.unit) * MAX_COLS + c4));
+        *reinterpret_cast<float4*>(lse_s + lb * MAX_COLS + c4) = val;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_lf(lb));
@@ -717,7 +755,7 @@ bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* pla
 
 cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv, int L,
                                  int d, int W, const ScorePlan& plan, float* vote, int* status,
-                                 int* counters, float2* partials, cudaStream_t stream,
+                                 int* counters, float2* partials, float* lse2, cudaStream_t stream,
                                  int* launches) {
   CUtensorMap tmK, tmQ;
   {
@@ -753,6 +791,7 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq
   a.pipelined = plan.pipelined;
   a.c2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
   a.partials = partials;
+  a.lse2 = lse2;
   a.counters = counters;
   a.status = status;
   a.vote = vote;
