@@ -177,7 +177,7 @@ __device__ __forceinline__ void for_each_item(const ScoreArgs& a, int cta, int G
 }
 
 // NCH = npad / 32: how many 32-column chunks of the accumulator a thread reads per tile.
-template <int D, int NCH>
+template <int D, int NCH, bool SPLIT>
 __global__ void __launch_bounds__(THREADS, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
              const ScoreArgs a) {
@@ -221,7 +221,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     }
     for (int b = 0; b < NBUF; ++b) {
       mbar_init(bar_tf(b), 1);
-      mbar_init(bar_te(b), 4);
+      mbar_init(bar_te(b), EPI_WARPS);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar_qf(b), 1);
@@ -353,6 +353,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     }
   } else if (warp < 2 + EPI_WARPS) {
     // ------------------------------------------------------------ softmax warps
+    // SPLIT: both warpgroups work on every tile, each on half of the accumulator columns
+    // (CPT columns per thread); the -lse values of a vote item then fit in registers.
+    // Otherwise the warpgroups alternate tiles and take all NPAD columns.
+    constexpr int CPT = SPLIT ? NPAD / 2 : NPAD;
+    constexpr int VCH = CPT / 32;
     const int wg = (warp - 2) >> 2;
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     const uint32_t lane_sel = static_cast<uint32_t>(32 * q) << 16;
@@ -360,8 +365,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     const int rep = rrow / NPAD;
     const int qcol = rrow - rep * NPAD;
     const int jmax = min(a.L - 1, a.n + (qcol % a.W));  // last key window row qcol % W sees
+    const int coff = SPLIT ? wg * CPT : 0;               // first accumulator column of this thread
     const bool w16 = (a.W & 15) == 0;
     const int gpw = a.W >> 4;  // 16-column groups per head (when W is a multiple of 16)
+    const uint32_t te_arrivals = SPLIT ? 1 : 2;          // the barrier expects 8 per tile
     int git = 0, nstat = 0, nvote = 0;
     for_each_item(a, cta, G, a.pipelined != 0, [&](const Item& it) {
       const int nt = it.t1 - it.t0;
@@ -372,33 +379,33 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         float m2 = -INFINITY;  // running max, log2 domain
         float l = 0.f;         // running sum of exp2(x - m2)
         for (int k = 0; k < nt; ++k, ++git) {
-          if ((git & 1) != wg) continue;
+          if (!SPLIT && (git & 1) != wg) continue;
           const int buf = git & (NBUF - 1);
           const uint32_t ub = (git / NBUF) & 1;
           if (!mbar_wait_warp(bar_tf(buf), ub, abort_s, WAIT_EPI_TMEM_FULL)) return false;
           tc_fence_after();
           const int key0 = tile_of(it, k) * TILE_KEYS;
-          // the whole slice of this thread's row: NPAD key columns
-          float v[NCH][32];
-          const uint32_t taddr = tmem_base + lane_sel + buf * 128 + rep * NPAD;
+          // this thread's slice of its window row: CPT key columns
+          float v[VCH][32];
+          const uint32_t taddr = tmem_base + lane_sel + buf * 128 + rep * NPAD + coff;
 #pragma unroll
-          for (int ch = 0; ch < NCH; ++ch) tmem_ld32(taddr + ch * 32, v[ch]);
+          for (int ch = 0; ch < VCH; ++ch) tmem_ld32(taddr + ch * 32, v[ch]);
           tmem_wait_ld();
           // the accumulator is in registers now: hand the buffer back to the MMA warp
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(bar_te(buf));
+          if (lane == 0) mbar_arrive_n(bar_te(buf), te_arrivals);
           if (key0 + TILE_KEYS - 1 > a.n) {  // tile touches the window or the prompt's end
-            const int kb = key0 + rep * NPAD;
+            const int kb = key0 + rep * NPAD + coff;
 #pragma unroll
-            for (int ch = 0; ch < NCH; ++ch)
+            for (int ch = 0; ch < VCH; ++ch)
 #pragma unroll
               for (int c = 0; c < 32; ++c)
                 v[ch][c] = (kb + ch * 32 + c <= jmax) ? v[ch][c] : -INFINITY;
           }
           float c0 = v[0][0], c1 = v[0][1], c2m = v[0][2], c3 = v[0][3];
 #pragma unroll
-          for (int ch = 0; ch < NCH; ++ch)
+          for (int ch = 0; ch < VCH; ++ch)
 #pragma unroll
             for (int c = (ch == 0 ? 4 : 0); c < 32; c += 4) {
               c0 = fmaxf(c0, v[ch][c + 0]);
@@ -411,7 +418,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           l *= ex2_approx(m2 - mnew);
           float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-          for (int ch = 0; ch < NCH; ++ch)
+          for (int ch = 0; ch < VCH; ++ch)
 #pragma unroll
             for (int c = 0; c < 32; c += 4) {
               s0 += ex2_approx(fmaf(v[ch][c + 0], a.c2, -mnew));
@@ -436,34 +443,52 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       const int lb = nvote % NLB;
       if (!mbar_wait_warp(bar_lf(lb), (nvote / NLB) & 1, abort_s, WAIT_LSE_FULL)) return false;
       const float* lse_b = lse_s + lb * MAX_COLS;
+      float lse_r[SPLIT ? VCH : 1][32];  // -lse of this thread's columns (SPLIT only)
+      if (SPLIT) {
+#pragma unroll
+        for (int ch = 0; ch < VCH; ++ch)
+#pragma unroll
+          for (int c4 = 0; c4 < 8; ++c4) {
+            const float4 z = *reinterpret_cast<const float4*>(lse_b + coff + ch * 32 + c4 * 4);
+            lse_r[ch][c4 * 4 + 0] = z.x;
+            lse_r[ch][c4 * 4 + 1] = z.y;
+            lse_r[ch][c4 * 4 + 2] = z.z;
+            lse_r[ch][c4 * 4 + 3] = z.w;
+          }
+      }
       for (int k = 0; k < nt; ++k, ++git) {
-        if ((git & 1) != wg) continue;
+        if (!SPLIT && (git & 1) != wg) continue;
         const int buf = git & (NBUF - 1);
         const uint32_t ub = (git / NBUF) & 1;
         if (!mbar_wait_warp(bar_tf(buf), ub, abort_s, WAIT_EPI_TMEM_FULL)) return false;
         tc_fence_after();
         const int j = tile_of(it, k) * TILE_KEYS + 32 * q + lane;
-        const uint32_t taddr = tmem_base + lane_sel + buf * 128;
-        // this key's logits against every window row of the unit
-        float v[NCH][32];
+        const uint32_t taddr = tmem_base + lane_sel + buf * 128 + coff;
+        // this key's logits against the window rows this thread covers
+        float v[VCH][32];
 #pragma unroll
-        for (int ch = 0; ch < NCH; ++ch) tmem_ld32(taddr + ch * 32, v[ch]);
+        for (int ch = 0; ch < VCH; ++ch) tmem_ld32(taddr + ch * 32, v[ch]);
         tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar_te(buf));
-        if (w16) {
+        if (lane == 0) mbar_arrive_n(bar_te(buf), te_arrivals);
+        if (SPLIT || w16) {
           // exp2(s * c2 - lse2) summed over each group of 16 columns, then groups -> heads
-          float g16[NCH * 2];
+          float g16[VCH * 2];
 #pragma unroll
-          for (int ch = 0; ch < NCH; ++ch)
+          for (int ch = 0; ch < VCH; ++ch)
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
-              const float4* nl = reinterpret_cast<const float4*>(lse_b + ch * 32 + hf * 16);
               float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
               for (int t4 = 0; t4 < 4; ++t4) {
-                const float4 z = nl[t4];
+                float4 z;
+                if (SPLIT) {
+                  z = make_float4(lse_r[ch][hf * 16 + 4 * t4 + 0], lse_r[ch][hf * 16 + 4 * t4 + 1],
+                                  lse_r[ch][hf * 16 + 4 * t4 + 2], lse_r[ch][hf * 16 + 4 * t4 + 3]);
+                } else {
+                  z = *reinterpret_cast<const float4*>(lse_b + ch * 32 + hf * 16 + 4 * t4);
+                }
                 a0 += ex2_approx(fmaf(v[ch][hf * 16 + 4 * t4 + 0], a.c2, z.x));
                 a1 += ex2_approx(fmaf(v[ch][hf * 16 + 4 * t4 + 1], a.c2, z.y));
                 a2 += ex2_approx(fmaf(v[ch][hf * 16 + 4 * t4 + 2], a.c2, z.z));
@@ -471,10 +496,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
               }
               g16[ch * 2 + hf] = (a0 + a1) + (a2 + a3);
             }
-          int hl = 0, left = gpw;
+          int hl = coff / a.W, left = gpw;  // SPLIT: coff is a multiple of W
           float acc = 0.f;
 #pragma unroll
-          for (int gi = 0; gi < NCH * 2; ++gi) {
+          for (int gi = 0; gi < VCH * 2; ++gi) {
             acc += g16[gi];
             if (--left == 0) {
               if (hl < a.hpu && j < a.n) a.vote[static_cast<size_t>(hq0 + hl) * a.n + j] = acc;
@@ -487,7 +512,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           int hl = 0, left = a.W;
           float acc = 0.f;
 #pragma unroll
-          for (int ch = 0; ch < NCH; ++ch)
+          for (int ch = 0; ch < VCH; ++ch)
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
               const int col = ch * 32 + c;
@@ -680,12 +705,12 @@ int sm_count() {
   return cached[dev];
 }
 
-template <int D, int NCH>
+template <int D, int NCH, bool SPLIT>
 cudaError_t run_scores(const CUtensorMap& tmK, const CUtensorMap& tmQ, const ScoreArgs& a,
                        int grid, cudaStream_t stream, int* launches) {
   static bool attr_done = false;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(score_kernel<D, NCH>,
+    cudaError_t e = cudaFuncSetAttribute(score_kernel<D, NCH, SPLIT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          Smem<D>::DYN_BYTES);
     if (e != cudaSuccess) return e;
@@ -695,7 +720,7 @@ cudaError_t run_scores(const CUtensorMap& tmK, const CUtensorMap& tmQ, const Sco
                      const_cast<ScoreArgs*>(&a)};
   // cooperative launch: every CTA is resident, so a CTA that waits for another CTA's
   // partial statistics cannot keep that CTA off the machine
-  cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(score_kernel<D, NCH>),
+  cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(score_kernel<D, NCH, SPLIT>),
                                               dim3(grid), dim3(THREADS), params,
                                               Smem<D>::DYN_BYTES, stream);
   if (e != cudaSuccess) return e;
@@ -798,14 +823,22 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq
   int grid = sm_count();
   if (grid > MAX_GRID) grid = MAX_GRID;
   const int nch = plan.npad >> 5;
+  // column-split epilogue when each warpgroup's half of the columns is whole heads
+  const bool split = nch >= 2 && (W % 16) == 0 && ((plan.npad / 2) % W) == 0;
   if (d == 64) {
-    if (nch == 1) return run_scores<64, 1>(tmK, tmQ, a, grid, stream, launches);
-    if (nch == 2) return run_scores<64, 2>(tmK, tmQ, a, grid, stream, launches);
-    return run_scores<64, 4>(tmK, tmQ, a, grid, stream, launches);
+    if (nch == 1) return run_scores<64, 1, false>(tmK, tmQ, a, grid, stream, launches);
+    if (nch == 2)
+      return split ? run_scores<64, 2, true>(tmK, tmQ, a, grid, stream, launches)
+                   : run_scores<64, 2, false>(tmK, tmQ, a, grid, stream, launches);
+    return split ? run_scores<64, 4, true>(tmK, tmQ, a, grid, stream, launches)
+                 : run_scores<64, 4, false>(tmK, tmQ, a, grid, stream, launches);
   }
-  if (nch == 1) return run_scores<128, 1>(tmK, tmQ, a, grid, stream, launches);
-  if (nch == 2) return run_scores<128, 2>(tmK, tmQ, a, grid, stream, launches);
-  return run_scores<128, 4>(tmK, tmQ, a, grid, stream, launches);
+  if (nch == 1) return run_scores<128, 1, false>(tmK, tmQ, a, grid, stream, launches);
+  if (nch == 2)
+    return split ? run_scores<128, 2, true>(tmK, tmQ, a, grid, stream, launches)
+                 : run_scores<128, 2, false>(tmK, tmQ, a, grid, stream, launches);
+  return split ? run_scores<128, 4, true>(tmK, tmQ, a, grid, stream, launches)
+               : run_scores<128, 4, false>(tmK, tmQ, a, grid, stream, launches);
 }
 
 }  // namespace snapkv
