@@ -19,8 +19,8 @@
 // kernel walks the phases  S(0), S(1), V(0), S(2), V(1), ...  so that the second sweep
 // over a wave's keys is served by L2 and the partials a vote phase needs were published
 // a whole phase earlier.  Within a phase the wave's tiles are split evenly over the CTAs.
-// One CTA per SM, launched cooperatively (all CTAs are resident, so waiting on another
-// CTA's partials cannot starve it).
+// One CTA per SM and no more CTAs than SMs, so all of them are resident and waiting on
+// another CTA's partials cannot starve it.
 //
 // Warp roles: warp 0 issues TMA loads (K tiles into a ring of stages, Q per work item
 // into two buffers), warp 1 issues tcgen05.mma into four TMEM accumulator buffers, warps
@@ -44,7 +44,8 @@ constexpr int STAGES = 4;
 constexpr int NBUF = 4;               // TMEM accumulator buffers of 128 columns
 constexpr int TMEM_COLS = 512;
 constexpr int SUBTILE_BYTES = 128 * 128;  // 128 rows x 64 bf16, 128-byte swizzled
-constexpr int THREADS = 352;          // producer, MMA, 8 softmax warps, book-keeper
+constexpr int THREADS = 384;          // producer, MMA, 8 softmax warps, book-keeper, 2nd MMA
+constexpr int MMA2_WARP = 11;
 constexpr int EPI_WARPS = 8;
 constexpr int NPB = 4;                // buffers for partial statistics (book-keeper queue)
 constexpr int NLB = 8;                // buffers for merged log-sum-exp rows
@@ -225,7 +226,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar_qf(b), 1);
-      mbar_init(bar_qe(b), 1);
+      mbar_init(bar_qe(b), 2);  // both MMA issuers release a Q buffer
     }
     for (int b = 0; b < NPB; ++b) {
       mbar_init(bar_pf(b), EPI_WARPS);
@@ -235,7 +236,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       mbar_init(bar_lf(b), 1);
       mbar_init(bar_le(b), EPI_WARPS);
     }
-    mbar_init(bar_drain, 1);
+    mbar_init(bar_drain, 2);
     *abort_s = 0;
     mbar_fence_init();
   }
@@ -309,8 +310,12 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
+  } else if (warp == 1 || warp == MMA2_WARP) {
+    // ------------------------------------------------------------ MMA issuers
+    // Two warps issue: one takes the even tiles, the other the odd ones.  A single
+    // thread cannot issue tcgen05.mma fast enough to keep the tensor pipe busy with
+    // 128 x 128 x 16 instructions.
+    const int mma_par = (warp == 1) ? 0 : 1;
     if (lane == 0) {
       const uint32_t idesc_s = umma_idesc_bf16(128, 128);
       const uint32_t idesc_v = umma_idesc_bf16(128, NPAD);
@@ -321,6 +326,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         ++nitem;
         const int nt = it.t1 - it.t0;
         for (int k = 0; k < nt; ++k, ++git) {
+          if ((git & 1) != mma_par) continue;
           const int s = git % STAGES;
           const uint32_t ph = (git / STAGES) & 1;
           const int buf = git & (NBUF - 1);
@@ -559,7 +565,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             for (int r = 0; r < REPS; ++r) {
               const int row = r * NPAD + c;
               const float2 p = ps[(w2 * 4 + (row >> 5)) * 32 + (row & 31)];
-              S += p.y * exp2f(p.x - M);
+              S += p.y * ex2_approx(p.x - M);
             }
           a.partials[(static_cast<size_t>(it.unit) * a.maxseg + it.slot) * MAX_COLS + c] =
               make_float2(M, S);
@@ -599,7 +605,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 #pragma unroll
                   for (int t = 0; t < 4; ++t) {
                     const float Mn = fmaxf(M[t], m[t]);
-                    S[t] = S[t] * exp2f(M[t] - Mn) + sv[t] * exp2f(m[t] - Mn);
+                    S[t] = S[t] * ex2_approx(M[t] - Mn) + sv[t] * ex2_approx(m[t] - Mn);
                     M[t] = Mn;
                   }
                 }
@@ -716,13 +722,12 @@ cudaError_t run_scores(const CUtensorMap& tmK, const CUtensorMap& tmQ, const Sco
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  void* params[3] = {const_cast<CUtensorMap*>(&tmK), const_cast<CUtensorMap*>(&tmQ),
-                     const_cast<ScoreArgs*>(&a)};
-  // cooperative launch: every CTA is resident, so a CTA that waits for another CTA's
-  // partial statistics cannot keep that CTA off the machine
-  cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(score_kernel<D, NCH, SPLIT>),
-                                              dim3(grid), dim3(THREADS), params,
-                                              Smem<D>::DYN_BYTES, stream);
+  // One CTA per SM (the shared-memory footprint allows no second one), grid no larger
+  // than the SM count: every CTA becomes resident as soon as the stream's earlier work
+  // has drained, so a CTA that waits for another CTA's partial statistics is waiting for
+  // a CTA that runs.  The waits are bounded in any case.
+  score_kernel<D, NCH, SPLIT><<<dim3(grid), dim3(THREADS), Smem<D>::DYN_BYTES, stream>>>(tmK, tmQ, a);
+  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   *launches += 1;
   return cudaSuccess;
