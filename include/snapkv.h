@@ -113,6 +113,28 @@ snapkv_status_t snapkv_pool_topk(const float* vote, int rows, int n,
                                  void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Pool + top-k without any caller-provided scratch.  The paper has no counterpart to this
+ * entry point: it exists for hosts that may not allocate device memory at the time of the
+ * call - an inference server whose memory pool was sized and frozen at start-up, code
+ * running between the launches of a latency-critical decode loop where a cudaMalloc would
+ * synchronise the device, or a plug-in that is handed tensors but no allocator.  Same
+ * inputs, outputs and result as snapkv_pool_topk; the per-vote keys go into a 16 MiB array
+ * that is part of the library image (every GPU that loads the library holds it until the
+ * process ends), so rows * n may not exceed SNAPKV_STATIC_MAX_KEYS: larger requests return
+ * SNAPKV_ERR_WORKSPACE and launch nothing.  The call allocates and frees nothing.
+ * The first call on each device looks up the array's device address (the device must be
+ * current); make that first call outside any stream capture.
+ * All calls share the one array and it keeps what the last call wrote.  Nothing in it has
+ * to start at zero - each launch writes every key before reading it - but two calls whose
+ * kernels overlap on the GPU (different streams, no dependency between them) race on it:
+ * order them.
+ */
+#define SNAPKV_STATIC_MAX_KEYS (4 * 1024 * 1024)
+snapkv_status_t snapkv_pool_topk_static(const float* vote, int rows, int n,
+                                        int pool_kernel, int pool_type, int ksel,
+                                        int32_t* out_idx, void* stream);
+
+/*
  * Step "gather + append" alone (Listing 1's gather and cat): with idx int32
  * [B, Hq, ksel] device (positions in [0, L - W)), writes per head the rows k[idx],
  * then the last W rows of k, to out_k [B, Hq, ksel + W, d]; same for v.

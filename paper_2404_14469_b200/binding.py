@@ -24,7 +24,7 @@ SYMBOLS = [
     "snapkv_status_string", "snapkv_out_rows", "snapkv_workspace_size", "snapkv_compress",
     "snapkv_window_scores", "snapkv_pool_topk_workspace_size", "snapkv_pool_topk", "snapkv_gather",
     "snapkv_host_staging_size", "snapkv_compress_host", "snapkv_device_status",
-    "snapkv_last_launch_count",
+    "snapkv_last_launch_count", "snapkv_pool_topk_static",
 ]
 
 _lib = None
@@ -59,6 +59,8 @@ def lib() -> ctypes.CDLL:
     L.snapkv_pool_topk_workspace_size.argtypes = [c_int, c_int]
     L.snapkv_pool_topk.restype = c_int
     L.snapkv_pool_topk.argtypes = [c_vp] + [c_int] * 5 + [c_vp, c_vp, c_sz, c_vp]
+    L.snapkv_pool_topk_static.restype = c_int
+    L.snapkv_pool_topk_static.argtypes = [c_vp] + [c_int] * 5 + [c_vp, c_vp]
     L.snapkv_gather.restype = c_int
     L.snapkv_gather.argtypes = [c_vp] * 3 + [c_int] * 7 + [c_vp] * 3
     L.snapkv_host_staging_size.restype = c_sz
@@ -177,6 +179,22 @@ def snapkv_pool_topk(vote, pool_kernel: int, pool_type: int, ksel: int, out_idx=
                                out_idx.data_ptr(), workspace.data_ptr() if workspace is not None else None,
                                workspace.numel() if workspace is not None else 0, _stream_ptr())
     _check(code, "snapkv_pool_topk")
+    return out_idx
+
+
+STATIC_MAX_KEYS = 4 * 1024 * 1024
+
+
+def snapkv_pool_topk_static(vote, pool_kernel: int, pool_type: int, ksel: int, out_idx):
+    """snapkv_pool_topk for callers that cannot allocate: the scratch is an array built
+    into the library (rows * n <= STATIC_MAX_KEYS).  `out_idx` (int32 [rows, ksel], CUDA)
+    must be passed in; this wrapper allocates nothing either."""
+    if not (vote.is_cuda and vote.dtype == torch.float32 and vote.is_contiguous() and vote.dim() == 2):
+        raise SnapKVError("vote must be a contiguous CUDA fp32 [rows, n] tensor")
+    rows, n = vote.shape
+    code = lib().snapkv_pool_topk_static(vote.data_ptr(), rows, n, pool_kernel, pool_type, ksel,
+                                         out_idx.data_ptr(), _stream_ptr())
+    _check(code, "snapkv_pool_topk_static")
     return out_idx
 
 

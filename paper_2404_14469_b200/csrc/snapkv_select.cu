@@ -14,6 +14,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "../../include/snapkv.h"
 #include "snapkv_internal.h"
 
 namespace snapkv {
@@ -387,3 +388,53 @@ cudaError_t launch_iota_idx(int32_t* out_idx, int rows, int n, int row_stride, c
 }
 
 }  // namespace snapkv
+
+// ---------------------------------------------------------------------------------------
+// Pool + top-k for callers that cannot hand the library any scratch memory.
+//
+// The generic kernel above keeps one 32-bit key per vote in global memory.  Here that
+// memory is a fixed array inside the library image instead of a caller buffer: 16 MiB that
+// every GPU which loads libsnapkv.so holds until the process exits.
+static __device__ __align__(256) uint32_t g_static_keys[SNAPKV_STATIC_MAX_KEYS];
+
+namespace snapkv {
+namespace {
+constexpr int MAX_DEVICES = 64;
+uint32_t* g_static_keys_addr[MAX_DEVICES] = {nullptr};
+
+// The array's name is only a handle on the host; the device address has to be asked for,
+// once per device, with that device current.
+snapkv_status_t static_keys_address(uint32_t** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return SNAPKV_ERR_CUDA;
+  if (g_static_keys_addr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_keys) != cudaSuccess || p == nullptr) return SNAPKV_ERR_CUDA;
+    g_static_keys_addr[dev] = static_cast<uint32_t*>(p);
+  }
+  *out = g_static_keys_addr[dev];
+  return SNAPKV_OK;
+}
+}  // namespace
+}  // namespace snapkv
+
+extern "C" snapkv_status_t snapkv_pool_topk_static(const float* vote, int rows, int n,
+                                                   int pool_kernel, int pool_type, int ksel,
+                                                   int32_t* out_idx, void* stream) {
+  using namespace snapkv;
+  if (rows < 1 || n < 1 || ksel < 1 || ksel > n || !vote || !out_idx) return SNAPKV_ERR_INVALID_ARG;
+  if (pool_kernel < 1 || (pool_kernel & 1) == 0) return SNAPKV_ERR_INVALID_ARG;
+  if (pool_type != SNAPKV_POOL_MAX && pool_type != SNAPKV_POOL_AVG) return SNAPKV_ERR_INVALID_ARG;
+  if (pool_kernel > 63) return SNAPKV_ERR_UNSUPPORTED;
+  // more keys than the built-in array holds: refuse before touching the device
+  if (static_cast<long long>(rows) * n > static_cast<long long>(SNAPKV_STATIC_MAX_KEYS))
+    return SNAPKV_ERR_WORKSPACE;
+  uint32_t* keys = nullptr;
+  const snapkv_status_t st = static_keys_address(&keys);
+  if (st != SNAPKV_OK) return st;
+  // Every key the kernel reads was written by the same launch, so nothing has to be
+  // cleared between calls; whatever the previous call left behind is overwritten or unused.
+  pool_topk_kernel<<<rows, SEL_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+      vote, n, pool_kernel, pool_type, ksel, out_idx, keys);
+  return cudaGetLastError() == cudaSuccess ? SNAPKV_OK : SNAPKV_ERR_CUDA;
+}
