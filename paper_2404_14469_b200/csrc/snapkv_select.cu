@@ -201,20 +201,37 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int base = threadIdx.x * ept;
 
-  // ---- 1. pooling over a rolling register window
+  // ---- 1. pooling
+  // The row is first copied into the key slots with coalesced loads (raw fp32 bits), then
+  // every thread pools its own positions in place over a rolling register window.  The
+  // values it needs from its neighbours' positions are saved before anybody overwrites.
   uint32_t kmin = 0xffffffffu, kmax = 0u;
   {
+    const int total = SEL_THREADS * ept;
+    for (int j = threadIdx.x; j < total; j += SEL_THREADS)
+      keys[key_slot(j)] = (j < n) ? __float_as_uint(__ldg(vrow + j)) : 0u;
+    __syncthreads();
     float w[2 * RMAX + 8];
+    float halo_r[RMAX > 0 ? RMAX : 1];
 #pragma unroll
-    for (int i = 0; i < 2 * RMAX; ++i) {
-      const int j = base - RMAX + i;
-      w[i] = (j >= 0 && j < n) ? __ldg(vrow + j) : 0.f;
+    for (int i = 0; i < RMAX; ++i) {
+      const int jl = base - RMAX + i;             // left neighbours
+      w[i] = (jl >= 0) ? __uint_as_float(keys[key_slot(jl)]) : 0.f;
+      const int jr = base + ept + i;              // right neighbours
+      halo_r[i] = (jr < total) ? __uint_as_float(keys[key_slot(jr)]) : 0.f;
     }
+#pragma unroll
+    for (int i = 0; i < RMAX; ++i) w[RMAX + i] = __uint_as_float(keys[key_slot(base + i)]);
+    __syncthreads();
     for (int sb = 0; sb < ept; sb += 8) {
+      const bool last = (sb + 8 == ept);
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        const int j = base + sb + RMAX + i;
-        w[2 * RMAX + i] = (j < n) ? __ldg(vrow + j) : 0.f;
+        // position base + sb + RMAX + i: own (not yet overwritten) or a saved right neighbour
+        float x;
+        if (i >= 8 - RMAX && last) x = halo_r[(i >= 8 - RMAX) ? i - (8 - RMAX) : 0];
+        else x = __uint_as_float(keys[key_slot(base + sb + RMAX + i)]);
+        w[2 * RMAX + i] = x;
       }
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
