@@ -106,35 +106,6 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def dist_setup(n_gpus):
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        import torch.distributed as dist
-
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
-    return rank, world, local
-
-
-def barrier(world):
-    if world > 1:
-        import torch.distributed as dist
-
-        dist.barrier()
-
-
-def max_over_ranks(x, world):
-    if world == 1:
-        return x
-    import torch.distributed as dist
-
-    t = torch.tensor([x], dtype=torch.float64, device="cuda" if torch.cuda.is_available() else "cpu")
-    dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    return float(t.item())
-
-
 # ------------------------------------------------------------------ reference arm (CPU oracle)
 def oracle_sample(w, budget, seconds_hint=15.0):
     """Time the CPU oracle, as it stands, on a bounded sample of one layer of the workload:
@@ -222,7 +193,13 @@ def main():
         run_reference(args, w, budget, int(os.environ.get("RANK", "0")),
                       int(os.environ.get("WORLD_SIZE", "1")))
         return
-    rank, world, local = dist_setup(args.gpus)
+    from paper_2404_14469_b200 import replicas
+
+    rank, world, local = replicas.init()
+    barrier = replicas.barrier
+
+    def max_over_ranks(x, world_):
+        return replicas.max_over_ranks(x, world_, device="cuda")
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the compression path has no CPU fallback")
@@ -242,7 +219,7 @@ def main():
     # every rank compresses its own batch of sequences)
     ins = []
     for layer in range(layers):
-        d = synth.make_layer(w, layer + 1000 * rank, device=str(dev))
+        d = synth.make_layer(w, layer + replicas.layer_seed_offset(rank), device=str(dev))
         ins.append((d["q_obs"], d["k"], d["v"]))
     out_k = [torch.empty(w.B, w.Hq, budget, w.d, dtype=torch.bfloat16, device=dev) for _ in range(layers)]
     out_v = [torch.empty_like(t) for t in out_k]
@@ -382,10 +359,7 @@ def main():
             "roofline": roofline, "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))
-    if world > 1:
-        import torch.distributed as dist
-
-        dist.destroy_process_group()
+    replicas.finish(world)
 
 
 if __name__ == "__main__":
