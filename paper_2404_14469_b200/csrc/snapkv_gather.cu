@@ -28,49 +28,48 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
                : "memory");
 }
 
-// VPR = 16-byte vectors per row.  One thread moves one vector of K and of V for
-// GATHER_UNROLL different rows, all loads issued before the first store.
+// VPR = 16-byte vectors per row.  blockIdx.y is the (batch, query head) pair, blockIdx.x a
+// block of RPB consecutive output rows of that head; one thread moves one vector of K and
+// of V for GATHER_UNROLL rows, all loads issued before the first store.  Index arithmetic
+// is 32-bit except for the final element offsets.
 template <int VPR>
 __global__ void __launch_bounds__(GATHER_THREADS)
 gather_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v,
               const int32_t* __restrict__ idx, int g, int L, int W, int ksel, int out_stride,
-              long long total_rows, uint4* __restrict__ out_k, uint4* __restrict__ out_v) {
+              uint4* __restrict__ out_k, uint4* __restrict__ out_v) {
+  constexpr int RPT = GATHER_THREADS / VPR;      // rows covered by the block per unrolled step
+  constexpr int RPB = RPT * GATHER_UNROLL;       // rows per block
   const int rows = ksel + W;
   const int n = L - W;
-  const long long vec0 = (static_cast<long long>(blockIdx.x) * GATHER_THREADS * GATHER_UNROLL) +
-                         threadIdx.x;
-  size_t src[GATHER_UNROLL], dst[GATHER_UNROLL];
+  const int bh = blockIdx.y;
+  const int vec = threadIdx.x % VPR;
+  const int t0 = blockIdx.x * RPB + threadIdx.x / VPR;
+  const size_t src_head = static_cast<size_t>(bh / g) * L * VPR + vec;
+  const size_t dst_head = static_cast<size_t>(bh) * out_stride * VPR + vec;
+  const int32_t* idx_head = idx ? idx + static_cast<size_t>(bh) * ksel : nullptr;
+  int pos[GATHER_UNROLL];
   bool ok[GATHER_UNROLL];
 #pragma unroll
   for (int uu = 0; uu < GATHER_UNROLL; ++uu) {
-    const long long gid = vec0 + static_cast<long long>(uu) * GATHER_THREADS;
-    const long long grow = gid / VPR;
-    const int vec = static_cast<int>(gid - grow * VPR);
-    ok[uu] = grow < total_rows;
-    src[uu] = dst[uu] = 0;
-    if (ok[uu]) {
-      const long long bh = grow / rows;
-      const int t = static_cast<int>(grow - bh * rows);
-      int pos;
-      if (t < ksel) pos = idx ? __ldg(idx + bh * ksel + t) : t;
-      else pos = n + (t - ksel);
-      const long long ukv = bh / g;
-      src[uu] = static_cast<size_t>((ukv * L + pos) * VPR + vec);
-      dst[uu] = static_cast<size_t>((bh * out_stride + t) * VPR + vec);
-    }
+    const int t = t0 + uu * RPT;
+    ok[uu] = t < rows;
+    pos[uu] = 0;
+    if (ok[uu]) pos[uu] = (t < ksel) ? (idx_head ? __ldg(idx_head + t) : t) : n + (t - ksel);
   }
   uint4 kk[GATHER_UNROLL], vv[GATHER_UNROLL];
 #pragma unroll
   for (int uu = 0; uu < GATHER_UNROLL; ++uu)
     if (ok[uu]) {
-      kk[uu] = ld_stream(k + src[uu]);
-      vv[uu] = ld_stream(v + src[uu]);
+      const size_t src = src_head + static_cast<size_t>(pos[uu]) * VPR;
+      kk[uu] = ld_stream(k + src);
+      vv[uu] = ld_stream(v + src);
     }
 #pragma unroll
   for (int uu = 0; uu < GATHER_UNROLL; ++uu)
     if (ok[uu]) {
-      st_stream(out_k + dst[uu], kk[uu]);
-      st_stream(out_v + dst[uu], vv[uu]);
+      const size_t dst = dst_head + static_cast<size_t>(t0 + uu * RPT) * VPR;
+      st_stream(out_k + dst, kk[uu]);
+      st_stream(out_v + dst, vv[uu]);
     }
 }
 
@@ -80,25 +79,34 @@ cudaError_t launch_gather(const void* k, const void* v, const int32_t* idx, int 
                           int L, int d, int W, int ksel, int out_rows_stride, void* out_k,
                           void* out_v, cudaStream_t stream, int* launches) {
   const int rows = ksel + W;
-  const long long total_rows = static_cast<long long>(B) * Hq * rows;
   const int vpr = d * 2 / 16;
-  const long long total_vec = total_rows * vpr;
-  const long long per_block = static_cast<long long>(GATHER_THREADS) * GATHER_UNROLL;
-  const long long blocks = (total_vec + per_block - 1) / per_block;
-  if (blocks <= 0) return cudaSuccess;
-  if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+  const int rpb = GATHER_THREADS / vpr * GATHER_UNROLL;
+  const long long heads = static_cast<long long>(B) * Hq;
+  if (rows <= 0 || heads <= 0) return cudaSuccess;
   const int g = Hq / Hkv;
   const uint4* kp = static_cast<const uint4*>(k);
   const uint4* vp = static_cast<const uint4*>(v);
   uint4* okp = static_cast<uint4*>(out_k);
   uint4* ovp = static_cast<uint4*>(out_v);
-  if (vpr == 16)
-    gather_kernel<16><<<static_cast<unsigned>(blocks), GATHER_THREADS, 0, stream>>>(
-        kp, vp, idx, g, L, W, ksel, out_rows_stride, total_rows, okp, ovp);
-  else
-    gather_kernel<8><<<static_cast<unsigned>(blocks), GATHER_THREADS, 0, stream>>>(
-        kp, vp, idx, g, L, W, ksel, out_rows_stride, total_rows, okp, ovp);
-  *launches += 1;
+  const unsigned gx = static_cast<unsigned>((rows + rpb - 1) / rpb);
+  // blockIdx.y is limited to 65535: go through the heads in slabs if there are more
+  // (each slab starts on a KV-head boundary so that bh / g stays right inside the kernel)
+  const long long slab = 65535 / g * g > 0 ? 65535 / g * g : g;
+  for (long long h0 = 0; h0 < heads; h0 += slab) {
+    const unsigned gy = static_cast<unsigned>(heads - h0 < slab ? heads - h0 : slab);
+    const int32_t* idx_s = idx ? idx + static_cast<size_t>(h0) * ksel : nullptr;
+    uint4* ok_s = okp + static_cast<size_t>(h0) * out_rows_stride * vpr;
+    uint4* ov_s = ovp + static_cast<size_t>(h0) * out_rows_stride * vpr;
+    const uint4* k_s = kp + static_cast<size_t>(h0 / g) * L * vpr;
+    const uint4* v_s = vp + static_cast<size_t>(h0 / g) * L * vpr;
+    if (vpr == 16)
+      gather_kernel<16><<<dim3(gx, gy), GATHER_THREADS, 0, stream>>>(k_s, v_s, idx_s, g, L, W, ksel,
+                                                                    out_rows_stride, ok_s, ov_s);
+    else
+      gather_kernel<8><<<dim3(gx, gy), GATHER_THREADS, 0, stream>>>(k_s, v_s, idx_s, g, L, W, ksel,
+                                                                   out_rows_stride, ok_s, ov_s);
+    *launches += 1;
+  }
   return cudaGetLastError();
 }
 
