@@ -44,8 +44,7 @@ constexpr int STAGES = 4;
 constexpr int NBUF = 4;               // TMEM accumulator buffers of 128 columns
 constexpr int TMEM_COLS = 512;
 constexpr int SUBTILE_BYTES = 128 * 128;  // 128 rows x 64 bf16, 128-byte swizzled
-constexpr int THREADS = 384;          // producer, MMA, 8 softmax warps, book-keeper, 2nd MMA
-constexpr int MMA2_WARP = 11;
+constexpr int THREADS = 352;          // producer, MMA, 8 softmax warps, book-keeper
 constexpr int EPI_WARPS = 8;
 constexpr int NPB = 4;                // buffers for partial statistics (book-keeper queue)
 constexpr int NLB = 8;                // buffers for merged log-sum-exp rows
@@ -193,6 +192,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   const uint32_t k_s = sbase + SM::OFF_K;
   const uint32_t bar0 = sbase + SM::OFF_BAR;
   auto q_s = [&](int b) { return sbase + SM::OFF_Q + b * SM::Q_BYTES; };
+  // Stages 2p and 2p+1 interleave so that each 64-element half of the head dimension is one
+  // 256-row tile across the pair: [half 0: stage 2p rows, stage 2p+1 rows][half 1: ...].
+  auto stage_addr = [&](int s, int sb) {
+    return k_s + (s >> 1) * (2 * SM::STAGE_BYTES) + sb * (2 * SUBTILE_BYTES) + (s & 1) * SUBTILE_BYTES;
+  };
   auto bar_full = [&](int s) { return bar0 + 8u * s; };
   auto bar_empty = [&](int s) { return bar0 + 8u * (STAGES + s); };
   auto bar_tf = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
@@ -226,7 +230,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar_qf(b), 1);
-      mbar_init(bar_qe(b), 2);  // both MMA issuers release a Q buffer
+      mbar_init(bar_qe(b), 1);
     }
     for (int b = 0; b < NPB; ++b) {
       mbar_init(bar_pf(b), EPI_WARPS);
@@ -236,7 +240,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       mbar_init(bar_lf(b), 1);
       mbar_init(bar_le(b), EPI_WARPS);
     }
-    mbar_init(bar_drain, 2);
+    mbar_init(bar_drain, 1);
     *abort_s = 0;
     mbar_fence_init();
   }
@@ -291,7 +295,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           mbar_expect_tx(bar_full(s), SM::STAGE_BYTES);
           const int key0 = tile_of(it, k) * TILE_KEYS;
           for (int sb = 0; sb < SUBT; ++sb)
-            tma_load_3d(k_s + s * SM::STAGE_BYTES + sb * SUBTILE_BYTES, &tmK, bar_full(s), sb * 64,
+            tma_load_3d(stage_addr(s, sb), &tmK, bar_full(s), sb * 64,
                         key0, ukv);
         }
         return true;
@@ -310,14 +314,15 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         }
       }
     }
-  } else if (warp == 1 || warp == MMA2_WARP) {
-    // ------------------------------------------------------------ MMA issuers
-    // Two warps issue: one takes the even tiles, the other the odd ones.  A single
-    // thread cannot issue tcgen05.mma fast enough to keep the tensor pipe busy with
-    // 128 x 128 x 16 instructions.
-    const int mma_par = (warp == 1) ? 0 : 1;
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    // The tensor pipe takes about as long for a 128 x N x 16 instruction with N <= 128 as
+    // for N = 256, so the statistics pass (keys on N) covers two key tiles per instruction
+    // whenever two tiles of an item sit in an aligned pair of stages: their accumulators
+    // are adjacent 128-column TMEM buffers, so the softmax warps see two ordinary tiles.
     if (lane == 0) {
       const uint32_t idesc_s = umma_idesc_bf16(128, 128);
+      const uint32_t idesc_s2 = umma_idesc_bf16(128, 256);
       const uint32_t idesc_v = umma_idesc_bf16(128, NPAD);
       int git = 0, nitem = 0;
       for_each_item(a, cta, G, a.pipelined != 0, [&](const Item& it) {
@@ -325,29 +330,37 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         if (!mbar_wait_thread(bar_qf(qb), (nitem >> 1) & 1, abort_s, WAIT_Q_FULL)) return false;
         ++nitem;
         const int nt = it.t1 - it.t0;
-        for (int k = 0; k < nt; ++k, ++git) {
-          if ((git & 1) != mma_par) continue;
+        for (int k = 0; k < nt;) {
           const int s = git % STAGES;
           const uint32_t ph = (git / STAGES) & 1;
           const int buf = git & (NBUF - 1);
           const uint32_t ub = (git / NBUF) & 1;
+          const bool pair = !it.vote && (git & 1) == 0 && k + 1 < nt;
           if (!mbar_wait_thread(bar_full(s), ph, abort_s, WAIT_MMA_FULL)) return false;
           if (!mbar_wait_thread(bar_te(buf), ub ^ 1, abort_s, WAIT_MMA_TMEM_EMPTY)) return false;
+          if (pair) {  // stage s + 1 and buffer buf + 1 are in the same round of their rings
+            if (!mbar_wait_thread(bar_full(s + 1), ph, abort_s, WAIT_MMA_FULL)) return false;
+            if (!mbar_wait_thread(bar_te(buf + 1), ub ^ 1, abort_s, WAIT_MMA_TMEM_EMPTY)) return false;
+          }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * 128;
 #pragma unroll
           for (int sb = 0; sb < SUBT; ++sb) {
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
-              const uint64_t kd =
-                  umma_desc_k128(k_s + s * SM::STAGE_BYTES + sb * SUBTILE_BYTES + kk * 32);
+              const uint64_t kd = umma_desc_k128(stage_addr(s, sb) + kk * 32);
               const uint64_t qd = umma_desc_k128(q_s(qb) + sb * SUBTILE_BYTES + kk * 32);
               if (it.vote) tc_mma_bf16(d_tmem, kd, qd, idesc_v, (sb | kk) != 0);
-              else tc_mma_bf16(d_tmem, qd, kd, idesc_s, (sb | kk) != 0);
+              else tc_mma_bf16(d_tmem, qd, kd, pair ? idesc_s2 : idesc_s, (sb | kk) != 0);
             }
           }
           tc_commit(bar_empty(s));
+          if (pair) tc_commit(bar_empty(s + 1));
           tc_commit(bar_tf(buf));
+          if (pair) tc_commit(bar_tf(buf + 1));
+          const int step = pair ? 2 : 1;
+          k += step;
+          git += step;
         }
         tc_commit(bar_qe(qb));  // the item's MMAs are the last readers of its Q buffer
         return true;
