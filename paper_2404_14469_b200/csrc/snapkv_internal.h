@@ -42,7 +42,7 @@ struct ScorePlan {
   int units_per_wave;
   int nwaves;
   int maxseg;       // partial-statistics slots per unit
-  int pipelined;    // phase order S0 S1 V0 S2 V1 ... (1) or S0 V0 S1 V1 ... (0)
+  int pipelined;    // how many waves the statistics pass runs ahead of the vote pass (>= 1)
 };
 
 struct WorkspaceLayout {

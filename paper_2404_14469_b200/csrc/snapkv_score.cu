@@ -46,8 +46,15 @@ constexpr int TMEM_COLS = 512;
 constexpr int SUBTILE_BYTES = 128 * 128;  // 128 rows x 64 bf16, 128-byte swizzled
 constexpr int THREADS = 352;          // producer, MMA, 8 softmax warps, book-keeper
 constexpr int EPI_WARPS = 8;
-constexpr int NPB = 4;                // buffers for partial statistics (book-keeper queue)
-constexpr int NLB = 8;                // buffers for merged log-sum-exp rows
+#ifndef WAVE_MIB
+#define WAVE_MIB 64
+#endif
+#ifndef WAVE_LAG
+#define WAVE_LAG 2
+#endif
+constexpr long long WAVE_BYTES = static_cast<long long>(WAVE_MIB) << 20;
+constexpr int NPB = 8;                // buffers for partial statistics (book-keeper queue)
+constexpr int NLB = 16;               // buffers for merged log-sum-exp rows
 
 struct ScoreArgs {
   int L, n, W;
@@ -56,7 +63,7 @@ struct ScoreArgs {
   int units, upw, nwaves;   // units per wave, number of waves
   int T1, T2;               // tiles per unit in the statistics / vote pass
   int maxseg;               // partial slots per unit
-  int pipelined;            // phase order S0 S1 V0 S2 V1 ... (else S0 V0 S1 V1 ...)
+  int pipelined;            // how many waves the statistics run ahead of the votes (>= 1)
   float c2;                 // log2(e) / sqrt(d)
   float2* partials;         // [units][maxseg][MAX_COLS] (max, sum) in the log2 domain
   float* lse2;              // [units][MAX_COLS] minus the merged log2-sum-exp per window row
@@ -132,20 +139,15 @@ __device__ __forceinline__ int cta_of_tile(long long x, long long TT, int G) {
 // Calls f(item) for every work item of this CTA in schedule order; stops when f
 // returns false.  All three warp roles walk the same list.
 template <typename F>
-__device__ __forceinline__ void for_each_item(const ScoreArgs& a, int cta, int G, bool pipelined,
+__device__ __forceinline__ void for_each_item(const ScoreArgs& a, int cta, int G, int lag,
                                               F&& f) {
-  const int nph = 2 * a.nwaves;
-  for (int p = 0; p < nph; ++p) {
+  // Phase order: statistics run `lag` waves ahead of votes: S(0) .. S(lag-1) V(0) S(lag)
+  // V(1) ...; lag = 1 is the plain order S(0) V(0) S(1) V(1) ...
+  int s_next = 0, v_next = 0;
+  while (v_next < a.nwaves) {
     int w, vote;
-    if (pipelined) {
-      if (p == 0) { w = 0; vote = 0; }
-      else if (p == nph - 1) { w = a.nwaves - 1; vote = 1; }
-      else if (p & 1) { w = (p + 1) >> 1; vote = 0; }
-      else { w = (p >> 1) - 1; vote = 1; }
-    } else {
-      w = p >> 1;
-      vote = p & 1;
-    }
+    if (s_next < a.nwaves && s_next - v_next < lag) { w = s_next++; vote = 0; }
+    else { w = v_next++; vote = 1; }
     const int u0 = w * a.upw;
     const int nu = min(a.upw, a.units - u0);
     const int T = vote ? a.T2 : a.T1;
@@ -256,7 +258,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   // tile visited at step k of an item: ascending, except that the sequential schedule
   // sweeps the vote pass backwards (the keys read last are the likeliest to be in L2)
   auto tile_of = [&](const Item& it, int k) {
-    return (it.vote && !a.pipelined) ? (it.t1 - 1 - k) : (it.t0 + k);
+    return (it.vote && a.pipelined == 1) ? (it.t1 - 1 - k) : (it.t0 + k);
   };
   auto first_head = [&](int unit, int* ukv) {
     *ukv = unit / a.sub_per_kv;
@@ -270,7 +272,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       tma_prefetch_desc(&tmQ);
       int git = 0;      // tiles issued so far (ring position)
       int nitem = 0;    // items started so far (Q buffer position)
-      for_each_item(a, cta, G, a.pipelined != 0, [&](const Item& it) {
+      for_each_item(a, cta, G, a.pipelined, [&](const Item& it) {
         int ukv;
         const int qrow0 = first_head(it.unit, &ukv) * a.W;
         const int qb = nitem & 1;
@@ -325,7 +327,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       const uint32_t idesc_s2 = umma_idesc_bf16(128, 256);
       const uint32_t idesc_v = umma_idesc_bf16(128, NPAD);
       int git = 0, nitem = 0;
-      for_each_item(a, cta, G, a.pipelined != 0, [&](const Item& it) {
+      for_each_item(a, cta, G, a.pipelined, [&](const Item& it) {
         const int qb = nitem & 1;
         if (!mbar_wait_thread(bar_qf(qb), (nitem >> 1) & 1, abort_s, WAIT_Q_FULL)) return false;
         ++nitem;
@@ -389,7 +391,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     const int gpw = a.W >> 4;  // 16-column groups per head (when W is a multiple of 16)
     const uint32_t te_arrivals = SPLIT ? 1 : 2;          // the barrier expects 8 per tile
     int git = 0, nstat = 0, nvote = 0;
-    for_each_item(a, cta, G, a.pipelined != 0, [&](const Item& it) {
+    for_each_item(a, cta, G, a.pipelined, [&](const Item& it) {
       const int nt = it.t1 - it.t0;
       int ukv;
       const int hq0 = first_head(it.unit, &ukv);
@@ -573,7 +575,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     // but the log-sum-exp of wave w is prepared right after wave w's statistics are
     // published, a whole phase before the softmax warps ask for it.
     int nstat = 0, nvote = 0;
-    for_each_item(a, cta, G, /*pipelined=*/false, [&](const Item& it) {
+    for_each_item(a, cta, G, /*lag=*/1, [&](const Item& it) {
       if (!it.vote) {
         // merge the replicas and the two warpgroups (fixed order), publish, count
         const int pb = nstat % NPB;
@@ -783,8 +785,8 @@ bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* pla
   // waves are live in L2 at a time, so a wave holds about 32 MiB of keys.  Units too big
   // for that take the sequential schedule, one unit per wave.
   const long long kbytes = static_cast<long long>(L) * d * 2;
-  long long kv_per_wave = (32ll << 20) / kbytes;
-  p.pipelined = kv_per_wave >= 1 ? 1 : 0;
+  long long kv_per_wave = (WAVE_BYTES) / kbytes;
+  p.pipelined = kv_per_wave >= 1 ? WAVE_LAG : 1;
   if (kv_per_wave < 1) kv_per_wave = 1;
   long long upw = kv_per_wave * p.sub_per_kv;
   // at most 128 units per wave: a CTA's share of a phase then spans few units, which
