@@ -184,6 +184,8 @@ pool_topk_kernel(const float* __restrict__ vote, int n, int pool_kernel, int poo
 // bank conflicts.  The first histogram pass bins (key - min) >> shift with the shift
 // chosen from the row's key range, so the bins are spread over the values that occur.
 __device__ __forceinline__ int key_slot(int j) { return j + (j >> 5); }
+constexpr int CAND_CAP = 2048;   // keys of the first-pass bin that are refined from a list
+constexpr int MASK_WORDS = 2;    // a thread owns at most 64 positions (SEL_SMEM_KEYS / SEL_THREADS = 48)
 
 template <int RMAX>
 __global__ void __launch_bounds__(SEL_THREADS, 1)
@@ -193,8 +195,10 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
   __shared__ int hist[NBINS];
   __shared__ int warp_sums[SEL_WARPS];
   __shared__ int scan_total;
-  __shared__ int sel_bin, sel_above;
+  __shared__ int sel_bin, sel_above, sel_count, ncand_s;
   __shared__ uint32_t red_min[SEL_WARPS], red_max[SEL_WARPS];
+  __shared__ uint32_t cand[CAND_CAP];
+  int ncand = 0;
 
   const int row = blockIdx.x;
   const float* vrow = vote + static_cast<size_t>(row) * n;
@@ -266,34 +270,50 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
   kmin = __reduce_min_sync(0xffffffffu, kmin);
   kmax = __reduce_max_sync(0xffffffffu, kmax);
 
-  // ---- 2. threshold: histogram passes over an ever narrower key range [lo, lo + width)
+  // ---- 2. threshold
+  // One histogram pass over all keys picks the bin that holds the ksel-th largest key.  A
+  // second sweep notes, per thread, which of its keys lie above that bin (kept for sure,
+  // one bit each) and which lie inside it, and copies the latter to a small candidate
+  // list; the remaining passes refine the threshold on that list alone.
   uint32_t lo = kmin;
   int krem = ksel;
   uint32_t T = kmin;
+  uint32_t m_gt[MASK_WORDS], m_in[MASK_WORDS];  // bit i: own key i above / inside the bin
+#pragma unroll
+  for (int wd = 0; wd < MASK_WORDS; ++wd) { m_gt[wd] = 0u; m_in[wd] = 0u; }
+  bool use_list = false;
   if (kmax != kmin) {
     const uint32_t range = kmax - kmin;
     int shift = 32 - __clz(range) - 11;
     if (shift < 0) shift = 0;
     uint32_t width_m1 = range;  // candidates are keys with key - lo <= width_m1
+    bool first = true;
 #pragma unroll 1
     for (;;) {
       for (int b = threadIdx.x; b < NBINS; b += SEL_THREADS) hist[b] = 0;
       __syncthreads();
-      int cur = -1, cnt = 0;
-      for (int i = 0; i < ept; ++i) {
-        const uint32_t key = keys[key_slot(base + i)];
-        const uint32_t rel = key - lo;
-        if (key >= lo && rel <= width_m1) {
-          const int b = static_cast<int>(rel >> shift);
-          if (b != cur) {
-            if (cnt) atomicAdd(&hist[cur], cnt);
-            cur = b;
-            cnt = 0;
+      if (!use_list) {
+        int cur = -1, cnt = 0;
+        for (int i = 0; i < ept; ++i) {
+          const uint32_t key = keys[key_slot(base + i)];
+          const uint32_t rel = key - lo;
+          if (key >= lo && rel <= width_m1) {
+            const int b = static_cast<int>(rel >> shift);
+            if (b != cur) {
+              if (cnt) atomicAdd(&hist[cur], cnt);
+              cur = b;
+              cnt = 0;
+            }
+            ++cnt;
           }
-          ++cnt;
+        }
+        if (cnt) atomicAdd(&hist[cur], cnt);
+      } else {
+        for (int c = threadIdx.x; c < ncand; c += SEL_THREADS) {
+          const uint32_t rel = cand[c] - lo;  // wraps to a huge value for keys below lo
+          if (rel <= width_m1) atomicAdd(&hist[rel >> shift], 1);
         }
       }
-      if (cnt) atomicAdd(&hist[cur], cnt);
       __syncthreads();
       int c0 = 0, c1 = 0;
       const int b0 = NBINS - 1 - 2 * static_cast<int>(threadIdx.x);
@@ -303,38 +323,80 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
       if (c0 > 0 && before < krem && krem <= before + c0) {
         sel_bin = b0;
         sel_above = before;
+        sel_count = c0;
       } else if (c1 > 0 && before + c0 < krem && krem <= before + c0 + c1) {
         sel_bin = b0 - 1;
         sel_above = before + c0;
+        sel_count = c1;
       }
+      if (threadIdx.x == 0) ncand_s = 0;
       __syncthreads();
       krem -= sel_above;
       lo += static_cast<uint32_t>(sel_bin) << shift;
+      const int in_bin = sel_count;
       const int done = (shift == 0);
       __syncthreads();
+      if (first) {
+        // classify own keys against the chosen bin; gather the bin's keys if they fit
+        first = false;
+        const uint32_t hi_m1 = done ? 0u : ((1u << shift) - 1u);
+        use_list = !done && in_bin <= CAND_CAP;
+        for (int i = 0; i < ept; ++i) {
+          const uint32_t key = keys[key_slot(base + i)];
+          const bool inb = key >= lo && key - lo <= hi_m1;
+          const bool gt = key >= lo && key - lo > hi_m1;
+          m_gt[i >> 5] |= static_cast<uint32_t>(gt) << (i & 31);
+          m_in[i >> 5] |= static_cast<uint32_t>(inb) << (i & 31);
+          if (inb && use_list) cand[atomicAdd(&ncand_s, 1)] = key;
+        }
+        __syncthreads();
+        ncand = ncand_s;
+      }
       if (done) break;
       width_m1 = (1u << shift) - 1u;
       shift = shift > 11 ? shift - 11 : 0;
     }
     T = lo;
+  } else {
+    // every key equals T
+#pragma unroll
+    for (int wd = 0; wd < MASK_WORDS; ++wd)
+      for (int i = wd * 32; i < min(ept, wd * 32 + 32); ++i)
+        if (base + i < n) m_in[wd] |= 1u << (i & 31);
   }
   const int need_eq = krem;
 
   // ---- 3. ordered compaction
+  // Keys inside the first bin are compared with the final threshold (few per thread), the
+  // rest is known from the bit masks; one block scan gives every thread its output offset.
+  uint32_t m_eq[MASK_WORDS];
   int cg = 0, ce = 0;
-  for (int i = 0; i < ept; ++i) {
-    const uint32_t key = keys[key_slot(base + i)];
-    cg += key > T;
-    ce += key == T;
+#pragma unroll
+  for (int wd = 0; wd < MASK_WORDS; ++wd) {
+    m_eq[wd] = 0u;
+    uint32_t rest = m_in[wd];
+    while (rest) {
+      const int i = wd * 32 + __ffs(rest) - 1;
+      rest &= rest - 1;
+      const uint32_t key = keys[key_slot(base + i)];
+      if (key > T) m_gt[wd] |= 1u << (i & 31);
+      else if (key == T) m_eq[wd] |= 1u << (i & 31);
+    }
+    cg += __popc(m_gt[wd]);
+    ce += __popc(m_eq[wd]);
   }
   const int packed = block_exclusive_scan((cg << 16) | ce, warp_sums, &scan_total);
   int eq_before = packed & 0xffff;
   int out_pos = (packed >> 16) + min(eq_before, need_eq);
   int32_t* orow = out_idx + static_cast<size_t>(row) * ksel;
-  if (cg + ce > 0) {
-    for (int i = 0; i < ept; ++i) {
-      const uint32_t key = keys[key_slot(base + i)];
-      if (key > T || (key == T && eq_before++ < need_eq)) orow[out_pos++] = base + i;
+#pragma unroll
+  for (int wd = 0; wd < MASK_WORDS; ++wd) {
+    uint32_t rest = m_gt[wd] | m_eq[wd];
+    while (rest) {
+      const int bit = __ffs(rest) - 1;
+      rest &= rest - 1;
+      const bool is_eq = (m_eq[wd] >> bit) & 1u;
+      if (!is_eq || eq_before++ < need_eq) orow[out_pos++] = base + wd * 32 + bit;
     }
   }
 }
