@@ -26,7 +26,7 @@ WorkspaceLayout make_layout(const ScorePlan& p, int B, int Hq, int n, bool need_
   const size_t row_bytes = sizeof(float) * static_cast<size_t>(B) * Hq * (n > 0 ? n : 0);
   if (need_vote) off = align_up(off + row_bytes, 256);
   w.off_pooled = off;
-  if (need_pooled) off = align_up(off + row_bytes, 256);
+  if (need_pooled) off = align_up(off + select_scratch_bytes(B * Hq, n), 256);
   w.total = off;
   return w;
 }
@@ -87,7 +87,7 @@ size_t snapkv_workspace_size(int B, int Hq, int Hkv, int L, int d, int W, int po
 
 size_t snapkv_pool_topk_workspace_size(int rows, int n) {
   if (rows < 1 || n < 1) return 0;
-  return select_needs_scratch(n) ? sizeof(float) * static_cast<size_t>(rows) * n : 0;
+  return select_scratch_bytes(rows, n);
 }
 
 snapkv_status_t snapkv_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv,
@@ -106,7 +106,9 @@ snapkv_status_t snapkv_window_scores(const void* q_obs, const void* k, int B, in
     return SNAPKV_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (cudaMemsetAsync(ws + w.off_status, 0, STATUS_BYTES, s) != cudaSuccess) return SNAPKV_ERR_CUDA;
+  // one memset clears the status block and the unit counters behind it
+  if (cudaMemsetAsync(ws + w.off_status, 0, w.off_partials - w.off_status, s) != cudaSuccess)
+    return SNAPKV_ERR_CUDA;
   int launches = 0;
   cudaError_t e = launch_window_scores(
       q_obs, k, B, Hq, Hkv, L, d, W, p, out_vote, reinterpret_cast<int*>(ws + w.off_status),
@@ -182,7 +184,9 @@ snapkv_status_t snapkv_compress(const void* q_obs, const void* k, const void* v,
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < w.total)
     return SNAPKV_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  if (cudaMemsetAsync(ws + w.off_status, 0, STATUS_BYTES, s) != cudaSuccess) return SNAPKV_ERR_CUDA;
+  // one memset clears the status block and the unit counters behind it
+  if (cudaMemsetAsync(ws + w.off_status, 0, w.off_partials - w.off_status, s) != cudaSuccess)
+    return SNAPKV_ERR_CUDA;
   float* vote = reinterpret_cast<float*>(ws + w.off_vote);
   const int ksel = budget - W;
   if (launch_window_scores(q_obs, k, B, Hq, Hkv, L, d, W, p, vote,

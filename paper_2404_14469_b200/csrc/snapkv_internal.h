@@ -53,15 +53,17 @@ bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* pla
 WorkspaceLayout make_layout(const ScorePlan& p, int B, int Hq, int n, bool need_vote,
                             bool need_pooled);
 bool select_needs_scratch(int n);
+size_t select_scratch_bytes(int rows, int n);  // 0 when the rows fit one CTA
 
-// Enqueue both scoring passes.  `vote` is fp32 [B*Hq, n].
+// Enqueue both scoring passes.  `vote` is fp32 [B*Hq, n].  `counters` must be zero when the
+// kernel starts (the callers clear it together with the status block).
 cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv, int L,
                                  int d, int W, const ScorePlan& plan, float* vote, int* status,
                                  int* counters, float2* partials, float* lse2, cudaStream_t stream,
                                  int* launches);
 
-// Pool + top-k over `rows` rows of fp32 votes.  `pooled_scratch` (fp32 [rows, n]) is
-// only touched when select_needs_scratch(n).
+// Pool + top-k over `rows` rows of fp32 votes.  `pooled_scratch` (select_scratch_bytes bytes)
+// is only touched when select_needs_scratch(n).
 cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel, int pool_type,
                              int ksel, int32_t* out_idx, float* pooled_scratch,
                              cudaStream_t stream, int* launches);

@@ -785,7 +785,9 @@ bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* pla
   // for that take the sequential schedule, one unit per wave.
   const long long kbytes = static_cast<long long>(L) * d * 2;
   long long kv_per_wave = (WAVE_BYTES) / kbytes;
-  p.pipelined = kv_per_wave >= 1 ? WAVE_LAG : 1;
+  // units bigger than a wave run one per wave: their second sweep comes from HBM, but the
+  // statistics of the next unit still hide the hand-over between the two passes
+  p.pipelined = WAVE_LAG;
   if (kv_per_wave < 1) kv_per_wave = 1;
   long long upw = kv_per_wave * p.sub_per_kv;
   // at most 128 units per wave: a CTA's share of a phase then spans few units, which
@@ -829,8 +831,6 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq
     cuuint32_t box[2] = {64, static_cast<cuuint32_t>(plan.npad)};
     if (!encode_map(&tmQ, q_obs, 2, dims, strides, box)) return cudaErrorInvalidValue;
   }
-  cudaError_t e = cudaMemsetAsync(counters, 0, sizeof(int) * plan.units, stream);
-  if (e != cudaSuccess) return e;
   ScoreArgs a;
   a.L = L;
   a.n = L - W;

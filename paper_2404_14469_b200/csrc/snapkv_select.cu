@@ -401,6 +401,220 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// Rows too long for one CTA's shared memory: the same radix select spread over many CTAs.
+// A row is cut into chunks of WIDE_CHUNK positions, one CTA each; histograms are built per
+// CTA in shared memory and added into a per-row histogram in global memory; a one-CTA-per-
+// row kernel picks the bin between the passes.  Keys live in global scratch:
+//   keys [rows][n] | hist [rows][NBINS] | state [rows][8] | counts [rows][nblk][2]
+// state: 0 prefix, 1 mask, 2 remaining rank.  Digits: 11, 11 and 10 bits from the top.
+constexpr int WIDE_THREADS = 256;
+constexpr int WIDE_EPT = 32;                            // positions per thread, contiguous
+constexpr int WIDE_CHUNK = WIDE_THREADS * WIDE_EPT;     // 8192 positions per CTA
+constexpr int WIDE_HALO = 31;                           // largest pooling radius
+
+struct WideBufs {
+  uint32_t* keys;
+  int* hist;
+  int* state;
+  int* counts;
+  int nblk;
+};
+
+__device__ __forceinline__ int wide_shift(int pass) { return pass == 0 ? 21 : (pass == 1 ? 10 : 0); }
+__device__ __forceinline__ int wide_bins(int pass) { return pass == 2 ? 1024 : 2048; }
+
+// Adds this CTA's keys that match the row's prefix into the row histogram (digit `pass`).
+__device__ __forceinline__ void wide_histogram(const uint32_t (&key_of_thread)[32], int valid, int pass,
+                                               uint32_t prefix, uint32_t mask, int* hist_s,
+                                               int* hist_g) {
+  const int shift = wide_shift(pass);
+  const uint32_t dmask = wide_bins(pass) - 1;
+  for (int b = threadIdx.x; b < NBINS; b += WIDE_THREADS) hist_s[b] = 0;
+  __syncthreads();
+  int cur = -1, cnt = 0;
+#pragma unroll
+  for (int i = 0; i < WIDE_EPT; ++i) {
+    const uint32_t key = key_of_thread[i];
+    if (i < valid && (key & mask) == prefix) {
+      const int b = static_cast<int>((key >> shift) & dmask);
+      if (b != cur) {
+        if (cnt) atomicAdd(&hist_s[cur], cnt);
+        cur = b;
+        cnt = 0;
+      }
+      ++cnt;
+    }
+  }
+  if (cnt) atomicAdd(&hist_s[cur], cnt);
+  __syncthreads();
+  for (int b = threadIdx.x; b < NBINS; b += WIDE_THREADS)
+    if (hist_s[b]) atomicAdd(&hist_g[b], hist_s[b]);
+}
+
+// Pooling of one chunk (staged through shared memory with its halo), keys to scratch, and
+// the first histogram pass.
+__global__ void __launch_bounds__(WIDE_THREADS)
+wide_pool_kernel(const float* __restrict__ vote, int n, int pool_kernel, int pool_type, WideBufs wb) {
+  __shared__ float raw[WIDE_CHUNK + 2 * WIDE_HALO + (WIDE_CHUNK + 2 * WIDE_HALO) / 32 + 1];
+  __shared__ int hist_s[NBINS];
+  const int row = blockIdx.y;
+  const int c0 = blockIdx.x * WIDE_CHUNK;
+  const int r = pool_kernel >> 1;
+  const float* vrow = vote + static_cast<size_t>(row) * n;
+  for (int t = threadIdx.x; t < WIDE_CHUNK + 2 * r; t += WIDE_THREADS) {
+    const int j = c0 - r + t;
+    raw[key_slot(t)] = (j >= 0 && j < n) ? __ldg(vrow + j) : 0.f;
+  }
+  __syncthreads();
+  uint32_t mine[WIDE_EPT];
+  const int base = threadIdx.x * WIDE_EPT;
+  int valid = n - (c0 + base);
+  valid = valid < 0 ? 0 : (valid > WIDE_EPT ? WIDE_EPT : valid);
+#pragma unroll
+  for (int i = 0; i < WIDE_EPT; ++i) {
+    float p = 0.f;  // votes are >= 0: zero is neutral for max and is the avg padding
+    for (int t = 0; t <= 2 * r; ++t) {
+      const float x = raw[key_slot(base + i + t)];
+      p = (pool_type == 0) ? fmaxf(p, x) : p + x;
+    }
+    if (pool_type != 0) p = p / static_cast<float>(pool_kernel);
+    mine[i] = float_to_key(p);
+  }
+  uint32_t* krow = wb.keys + static_cast<size_t>(row) * n + c0 + base;
+#pragma unroll
+  for (int i = 0; i < WIDE_EPT; ++i)
+    if (i < valid) krow[i] = mine[i];
+  wide_histogram(mine, valid, 0, 0u, 0u, hist_s, wb.hist + static_cast<size_t>(row) * NBINS);
+}
+
+// One CTA per row: walk the row histogram from the top, fix the next digit of the
+// threshold, clear the histogram for the next pass.
+__global__ void __launch_bounds__(SEL_THREADS)
+wide_pick_kernel(int pass, int ksel, WideBufs wb) {
+  __shared__ int warp_sums[SEL_WARPS];
+  __shared__ int scan_total;
+  const int row = blockIdx.x;
+  int* hist = wb.hist + static_cast<size_t>(row) * NBINS;
+  int* st = wb.state + row * 8;
+  const int nb = wide_bins(pass);
+  const int krem = pass == 0 ? ksel : st[2];
+  const uint32_t prefix = pass == 0 ? 0u : static_cast<uint32_t>(st[0]);
+  const uint32_t mask = pass == 0 ? 0u : static_cast<uint32_t>(st[1]);
+  int c0 = 0, c1 = 0;
+  const int b0 = nb - 1 - 2 * static_cast<int>(threadIdx.x);
+  if (b0 >= 0) c0 = hist[b0];
+  if (b0 - 1 >= 0) c1 = hist[b0 - 1];
+  const int before = block_exclusive_scan(c0 + c1, warp_sums, &scan_total);
+  int bin = -1, above = 0;
+  if (c0 > 0 && before < krem && krem <= before + c0) { bin = b0; above = before; }
+  else if (c1 > 0 && before + c0 < krem && krem <= before + c0 + c1) { bin = b0 - 1; above = before + c0; }
+  __syncthreads();  // every thread has read the state and its bins
+  if (bin >= 0) {
+    const int shift = wide_shift(pass);
+    st[0] = static_cast<int>(prefix | (static_cast<uint32_t>(bin) << shift));
+    st[1] = static_cast<int>(mask | (static_cast<uint32_t>(nb - 1) << shift));
+    st[2] = krem - above;
+  }
+  for (int b = threadIdx.x; b < NBINS; b += SEL_THREADS) hist[b] = 0;
+}
+
+__global__ void __launch_bounds__(WIDE_THREADS)
+wide_hist_kernel(int n, int pass, WideBufs wb) {
+  __shared__ int hist_s[NBINS];
+  const int row = blockIdx.y;
+  const int base = blockIdx.x * WIDE_CHUNK + threadIdx.x * WIDE_EPT;
+  int valid = n - base;
+  valid = valid < 0 ? 0 : (valid > WIDE_EPT ? WIDE_EPT : valid);
+  uint32_t mine[WIDE_EPT];
+  const uint32_t* krow = wb.keys + static_cast<size_t>(row) * n + base;
+#pragma unroll
+  for (int i = 0; i < WIDE_EPT; ++i) mine[i] = (i < valid) ? krow[i] : 0u;
+  const int* st = wb.state + row * 8;
+  wide_histogram(mine, valid, pass, static_cast<uint32_t>(st[0]), static_cast<uint32_t>(st[1]),
+                 hist_s, wb.hist + static_cast<size_t>(row) * NBINS);
+}
+
+// Per chunk: how many keys are above the threshold and how many equal it.
+__global__ void __launch_bounds__(WIDE_THREADS)
+wide_count_kernel(int n, WideBufs wb) {
+  __shared__ int sg, se;
+  const int row = blockIdx.y;
+  if (threadIdx.x == 0) { sg = 0; se = 0; }
+  __syncthreads();
+  const uint32_t T = static_cast<uint32_t>(wb.state[row * 8 + 0]);
+  const int base = blockIdx.x * WIDE_CHUNK + threadIdx.x * WIDE_EPT;
+  const uint32_t* krow = wb.keys + static_cast<size_t>(row) * n + base;
+  int cg = 0, ce = 0;
+  for (int i = 0; i < WIDE_EPT && base + i < n; ++i) {
+    const uint32_t key = krow[i];
+    cg += key > T;
+    ce += key == T;
+  }
+  cg = __reduce_add_sync(0xffffffffu, cg);
+  ce = __reduce_add_sync(0xffffffffu, ce);
+  if ((threadIdx.x & 31) == 0) { atomicAdd(&sg, cg); atomicAdd(&se, ce); }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int* c = wb.counts + (static_cast<size_t>(row) * wb.nblk + blockIdx.x) * 2;
+    c[0] = sg;
+    c[1] = se;
+  }
+}
+
+// Ordered compaction: every key above the threshold, and the lowest-position keys equal
+// to it until ksel positions are out, in ascending position.
+__global__ void __launch_bounds__(WIDE_THREADS)
+wide_write_kernel(int n, int ksel, int32_t* __restrict__ out_idx, WideBufs wb) {
+  __shared__ int warp_sums[SEL_WARPS];
+  __shared__ int scan_total;
+  const int row = blockIdx.y;
+  const uint32_t T = static_cast<uint32_t>(wb.state[row * 8 + 0]);
+  const int need_eq = wb.state[row * 8 + 2];
+  // keys selected in the chunks before this one (a short serial sum)
+  int gt_before = 0, eq_before = 0;
+  const int* c = wb.counts + static_cast<size_t>(row) * wb.nblk * 2;
+  for (int b = 0; b < static_cast<int>(blockIdx.x); ++b) {
+    gt_before += c[2 * b];
+    eq_before += c[2 * b + 1];
+  }
+  const int base = blockIdx.x * WIDE_CHUNK + threadIdx.x * WIDE_EPT;
+  const uint32_t* krow = wb.keys + static_cast<size_t>(row) * n + base;
+  uint32_t m_gt = 0u, m_eq = 0u;
+  for (int i = 0; i < WIDE_EPT && base + i < n; ++i) {
+    const uint32_t key = krow[i];
+    m_gt |= static_cast<uint32_t>(key > T) << i;
+    m_eq |= static_cast<uint32_t>(key == T) << i;
+  }
+  // block scan over 256 threads: block_exclusive_scan expects SEL_WARPS warp slots
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x < SEL_WARPS) warp_sums[threadIdx.x] = 0;
+  __syncthreads();
+  int x = (__popc(m_gt) << 16) | __popc(m_eq);
+  int inc = x;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += y;
+  }
+  if (lane == 31) warp_sums[warp] = inc;
+  __syncthreads();
+  int wpre = 0;
+  for (int w2 = 0; w2 < warp; ++w2) wpre += warp_sums[w2];
+  const int packed = wpre + inc - x;
+  (void)scan_total;
+  int eq_seen = eq_before + (packed & 0xffff);
+  int out_pos = gt_before + (packed >> 16) + min(eq_seen, need_eq);
+  int32_t* orow = out_idx + static_cast<size_t>(row) * ksel;
+  uint32_t rest = m_gt | m_eq;
+  while (rest) {
+    const int bit = __ffs(rest) - 1;
+    rest &= rest - 1;
+    const bool is_eq = (m_eq >> bit) & 1u;
+    if (!is_eq || eq_seen++ < need_eq) orow[out_pos++] = base + bit;
+  }
+}
+
 __global__ void iota_kernel(int32_t* out, int rows, int n, int row_stride) {
   const long long total = static_cast<long long>(rows) * n;
   for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
@@ -417,6 +631,16 @@ static inline int key_slot_host(int j) { return j + (j >> 5); }
 constexpr int FAST_SMEM_BYTES = (SEL_SMEM_KEYS + SEL_SMEM_KEYS / 32 + 64) * 4;
 
 bool select_needs_scratch(int n) { return n > SEL_SMEM_KEYS; }
+
+static inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+static inline int wide_nblk(int n) { return (n + WIDE_CHUNK - 1) / WIDE_CHUNK; }
+
+// Scratch of the many-CTA path: keys | row histograms | row state | chunk counts.
+size_t select_scratch_bytes(int rows, int n) {
+  if (!select_needs_scratch(n)) return 0;
+  const size_t r = static_cast<size_t>(rows);
+  return up256(r * n * 4) + up256(r * NBINS * 4) + up256(r * 8 * 4) + up256(r * wide_nblk(n) * 2 * 4);
+}
 
 cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel, int pool_type,
                              int ksel, int32_t* out_idx, float* pooled_scratch,
@@ -447,12 +671,36 @@ cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel
     *launches += 1;
     return cudaGetLastError();
   }
-  const bool scratch = select_needs_scratch(n);
-  const size_t dyn = scratch ? 0 : static_cast<size_t>(n) * 4;
-  pool_topk_kernel<<<rows, SEL_THREADS, dyn, stream>>>(
-      vote, n, pool_kernel, pool_type, ksel, out_idx,
-      scratch ? reinterpret_cast<uint32_t*>(pooled_scratch) : nullptr);
-  *launches += 1;
+  if (!select_needs_scratch(n)) {  // fits one CTA, but the radius is beyond the fast path
+    pool_topk_kernel<<<rows, SEL_THREADS, static_cast<size_t>(n) * 4, stream>>>(
+        vote, n, pool_kernel, pool_type, ksel, out_idx, nullptr);
+    *launches += 1;
+    return cudaGetLastError();
+  }
+  // long rows: many CTAs per row, state in global scratch
+  WideBufs wb;
+  uint8_t* p = reinterpret_cast<uint8_t*>(pooled_scratch);
+  const size_t nr = static_cast<size_t>(rows);
+  wb.nblk = wide_nblk(n);
+  wb.keys = reinterpret_cast<uint32_t*>(p);
+  p += up256(nr * n * 4);
+  wb.hist = reinterpret_cast<int*>(p);
+  p += up256(nr * NBINS * 4);
+  wb.state = reinterpret_cast<int*>(p);
+  p += up256(nr * 8 * 4);
+  wb.counts = reinterpret_cast<int*>(p);
+  cudaError_t e = cudaMemsetAsync(wb.hist, 0, up256(nr * NBINS * 4), stream);
+  if (e != cudaSuccess) return e;
+  const dim3 grid(wb.nblk, rows);
+  wide_pool_kernel<<<grid, WIDE_THREADS, 0, stream>>>(vote, n, pool_kernel, pool_type, wb);
+  wide_pick_kernel<<<rows, SEL_THREADS, 0, stream>>>(0, ksel, wb);
+  wide_hist_kernel<<<grid, WIDE_THREADS, 0, stream>>>(n, 1, wb);
+  wide_pick_kernel<<<rows, SEL_THREADS, 0, stream>>>(1, ksel, wb);
+  wide_hist_kernel<<<grid, WIDE_THREADS, 0, stream>>>(n, 2, wb);
+  wide_pick_kernel<<<rows, SEL_THREADS, 0, stream>>>(2, ksel, wb);
+  wide_count_kernel<<<grid, WIDE_THREADS, 0, stream>>>(n, wb);
+  wide_write_kernel<<<grid, WIDE_THREADS, 0, stream>>>(n, ksel, out_idx, wb);
+  *launches += 8;
   return cudaGetLastError();
 }
 

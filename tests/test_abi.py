@@ -60,7 +60,8 @@ def test_workspace_size(L):
                 (1, 4, 4, 100, 64, 200, 7, 0, 300), (1, 4, 4, 100, 64, 101, 7, 0, 300)]:
         assert sk.snapkv_workspace_size(*bad) == 0, bad
     assert sk.lib().snapkv_pool_topk_workspace_size(4, 1000) == 0
-    assert sk.lib().snapkv_pool_topk_workspace_size(4, 100000) == 4 * 100000 * 4
+    # long rows: one key per vote plus small per-row histograms and counters
+    assert 4 * 100000 * 4 < sk.lib().snapkv_pool_topk_workspace_size(4, 100000) < 4 * 100000 * 4 + (1 << 16)
     assert sk.snapkv_host_staging_size(1, 4, 4, 1024, 64, 32, 7, 0, 256) > 2 * 4 * 1024 * 64 * 2
 
 
