@@ -25,6 +25,10 @@ if ROOT not in sys.path:
 
 import torch  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries
+# (profiles/): (stage, workload id) -> bytes; None for anything not captured
+NCU_TRAFFIC = {("score", 2): 549.9e6, ("gather", 2): 338.2e6}
+
 METRIC = "prompt_tokens_compressed_per_s"
 UNIT = "prompt tokens/s"
 
@@ -299,7 +303,7 @@ def main():
         "bound": "hbm", "kernel": {"score": "score_kernel (statistics + vote passes)",
                                     "gather": "gather_kernel"}[dom],
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "peak_kind": f"of {peak_kind}", "traffic": None,
+        "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC.get((dom, w.wid)),
         "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": stage_ms[dom],
         "stage_ms_per_layer": stage_ms,
         "whole_step": {"algorithmic_bytes_per_layer": ab["total"], "ms_per_layer": ms_layer,
