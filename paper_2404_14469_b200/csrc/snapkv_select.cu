@@ -481,10 +481,14 @@ wide_pool_kernel(const float* __restrict__ vote, int n, int pool_kernel, int poo
     if (pool_type != 0) p = p / static_cast<float>(pool_kernel);
     mine[i] = float_to_key(p);
   }
-  uint32_t* krow = wb.keys + static_cast<size_t>(row) * n + c0 + base;
+  // keys go out through shared memory so that the global stores are coalesced
+  __syncthreads();  // everybody is done reading the raw votes
+  uint32_t* stage = reinterpret_cast<uint32_t*>(raw);
 #pragma unroll
-  for (int i = 0; i < WIDE_EPT; ++i)
-    if (i < valid) krow[i] = mine[i];
+  for (int i = 0; i < WIDE_EPT; ++i) stage[key_slot(base + i)] = mine[i];
+  __syncthreads();
+  uint32_t* krow = wb.keys + static_cast<size_t>(row) * n + c0;
+  for (int t = threadIdx.x; t < WIDE_CHUNK && c0 + t < n; t += WIDE_THREADS) krow[t] = stage[key_slot(t)];
   wide_histogram(mine, valid, 0, 0u, 0u, hist_s, wb.hist + static_cast<size_t>(row) * NBINS);
 }
 
@@ -523,16 +527,28 @@ __global__ void __launch_bounds__(WIDE_THREADS)
 wide_hist_kernel(int n, int pass, WideBufs wb) {
   __shared__ int hist_s[NBINS];
   const int row = blockIdx.y;
-  const int base = blockIdx.x * WIDE_CHUNK + threadIdx.x * WIDE_EPT;
-  int valid = n - base;
-  valid = valid < 0 ? 0 : (valid > WIDE_EPT ? WIDE_EPT : valid);
-  uint32_t mine[WIDE_EPT];
-  const uint32_t* krow = wb.keys + static_cast<size_t>(row) * n + base;
-#pragma unroll
-  for (int i = 0; i < WIDE_EPT; ++i) mine[i] = (i < valid) ? krow[i] : 0u;
+  // lane-strided reads (coalesced); the order of the keys does not matter here.  Only keys
+  // that match the row's prefix count, and those are few after the first pass.
+  const int c0 = blockIdx.x * WIDE_CHUNK;
+  const uint32_t* krow = wb.keys + static_cast<size_t>(row) * n + c0;
   const int* st = wb.state + row * 8;
-  wide_histogram(mine, valid, pass, static_cast<uint32_t>(st[0]), static_cast<uint32_t>(st[1]),
-                 hist_s, wb.hist + static_cast<size_t>(row) * NBINS);
+  const uint32_t prefix = static_cast<uint32_t>(st[0]), mask = static_cast<uint32_t>(st[1]);
+  const int shift = wide_shift(pass);
+  const uint32_t dmask = wide_bins(pass) - 1;
+  for (int b = threadIdx.x; b < NBINS; b += WIDE_THREADS) hist_s[b] = 0;
+  __syncthreads();
+#pragma unroll 8
+  for (int i = 0; i < WIDE_EPT; ++i) {
+    const int t = i * WIDE_THREADS + threadIdx.x;
+    if (c0 + t < n) {
+      const uint32_t key = krow[t];
+      if ((key & mask) == prefix) atomicAdd(&hist_s[(key >> shift) & dmask], 1);
+    }
+  }
+  __syncthreads();
+  int* hist_g = wb.hist + static_cast<size_t>(row) * NBINS;
+  for (int b = threadIdx.x; b < NBINS; b += WIDE_THREADS)
+    if (hist_s[b]) atomicAdd(&hist_g[b], hist_s[b]);
 }
 
 // Per chunk: how many keys are above the threshold and how many equal it.
@@ -543,13 +559,17 @@ wide_count_kernel(int n, WideBufs wb) {
   if (threadIdx.x == 0) { sg = 0; se = 0; }
   __syncthreads();
   const uint32_t T = static_cast<uint32_t>(wb.state[row * 8 + 0]);
-  const int base = blockIdx.x * WIDE_CHUNK + threadIdx.x * WIDE_EPT;
-  const uint32_t* krow = wb.keys + static_cast<size_t>(row) * n + base;
+  const int c0 = blockIdx.x * WIDE_CHUNK;
+  const uint32_t* krow = wb.keys + static_cast<size_t>(row) * n + c0;
   int cg = 0, ce = 0;
-  for (int i = 0; i < WIDE_EPT && base + i < n; ++i) {
-    const uint32_t key = krow[i];
-    cg += key > T;
-    ce += key == T;
+#pragma unroll 8
+  for (int i = 0; i < WIDE_EPT; ++i) {
+    const int t = i * WIDE_THREADS + threadIdx.x;
+    if (c0 + t < n) {
+      const uint32_t key = krow[t];
+      cg += key > T;
+      ce += key == T;
+    }
   }
   cg = __reduce_add_sync(0xffffffffu, cg);
   ce = __reduce_add_sync(0xffffffffu, ce);
@@ -578,13 +598,23 @@ wide_write_kernel(int n, int ksel, int32_t* __restrict__ out_idx, WideBufs wb) {
     gt_before += c[2 * b];
     eq_before += c[2 * b + 1];
   }
-  const int base = blockIdx.x * WIDE_CHUNK + threadIdx.x * WIDE_EPT;
-  const uint32_t* krow = wb.keys + static_cast<size_t>(row) * n + base;
+  __shared__ uint32_t stage[WIDE_CHUNK + WIDE_CHUNK / 32 + 1];
+  const int c0 = blockIdx.x * WIDE_CHUNK;
+  {
+    const uint32_t* kin = wb.keys + static_cast<size_t>(row) * n + c0;
+    for (int t = threadIdx.x; t < WIDE_CHUNK; t += WIDE_THREADS)
+      stage[key_slot(t)] = (c0 + t < n) ? kin[t] : 0u;
+  }
+  __syncthreads();
+  const int lbase = threadIdx.x * WIDE_EPT;
+  const int base = c0 + lbase;
   uint32_t m_gt = 0u, m_eq = 0u;
-  for (int i = 0; i < WIDE_EPT && base + i < n; ++i) {
-    const uint32_t key = krow[i];
-    m_gt |= static_cast<uint32_t>(key > T) << i;
-    m_eq |= static_cast<uint32_t>(key == T) << i;
+#pragma unroll
+  for (int i = 0; i < WIDE_EPT; ++i) {
+    const uint32_t key = stage[key_slot(lbase + i)];
+    const bool in = base + i < n;
+    m_gt |= static_cast<uint32_t>(in && key > T) << i;
+    m_eq |= static_cast<uint32_t>(in && key == T) << i;
   }
   // block scan over 256 threads: block_exclusive_scan expects SEL_WARPS warp slots
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
