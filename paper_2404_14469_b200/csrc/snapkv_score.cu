@@ -25,9 +25,12 @@
 // Warp roles: warp 0 issues TMA loads (K tiles into a ring of stages, Q per work item
 // into two buffers), warp 1 issues tcgen05.mma into four TMEM accumulator buffers, warps
 // 2-9 (two warpgroups, alternating tiles) read the accumulators back with tcgen05.ld and
-// do the fp32 softmax arithmetic, warp 10 is the book-keeper: it merges and publishes the
-// partial statistics the softmax warps leave in shared memory, and prepares the merged
-// log-sum-exp of the next vote item while the softmax warps are still busy.
+// do the fp32 softmax arithmetic, warps 10 and 11 are the book-keepers: warp 10 merges and
+// publishes the partial statistics the softmax warps leave in shared memory, warp 11
+// fetches the merged log-sum-exp of the coming vote items while the softmax warps are
+// still busy.  The single-thread roles (TMA and MMA issue) are entered through elect.sync:
+// the compiler then keeps descriptors and addresses in uniform registers, which cut the
+// time per tcgen05.mma issue by about a third against a lane-index test.
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <math.h>
@@ -44,7 +47,7 @@ constexpr int STAGES = 4;
 constexpr int NBUF = 4;               // TMEM accumulator buffers of 128 columns
 constexpr int TMEM_COLS = 512;
 constexpr int SUBTILE_BYTES = 128 * 128;  // 128 rows x 64 bf16, 128-byte swizzled
-constexpr int THREADS = 352;          // producer, MMA, 8 softmax warps, book-keeper
+constexpr int THREADS = 384;          // producer, MMA, 8 softmax warps, publisher, lse fetcher
 constexpr int EPI_WARPS = 8;
 #ifndef WAVE_MIB
 #define WAVE_MIB 64
@@ -269,7 +272,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    if (elect_one()) {
       tma_prefetch_desc(&tmK);
       tma_prefetch_desc(&tmQ);
       int git = 0;      // tiles issued so far (ring position)
@@ -324,7 +327,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     // for N = 256, so the statistics pass (keys on N) covers two key tiles per instruction
     // whenever two tiles of an item sit in an aligned pair of stages: their accumulators
     // are adjacent 128-column TMEM buffers, so the softmax warps see two ordinary tiles.
-    if (lane == 0) {
+    if (elect_one()) {
       const uint32_t idesc_s = umma_idesc_bf16(128, 128);
       const uint32_t idesc_s2 = umma_idesc_bf16(128, 256);
       const uint32_t idesc_v = umma_idesc_bf16(128, NPAD);
@@ -568,13 +571,15 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       return true;
     });
   } else {
-    // ------------------------------------------------------------ book-keeper warp
-    // It walks the waves in the order S(0) V(0) S(1) V(1) ...: the same statistics items
-    // and the same vote items as the other roles, each kind in the same relative order,
-    // but the log-sum-exp of wave w is prepared right after wave w's statistics are
-    // published, a whole phase before the softmax warps ask for it.
+    // ------------------------------------------------------------ book-keeper warps
+    // Warp 10 publishes this CTA's statistics partials (and merges a unit when it was the
+    // last to publish); warp 11 fetches the merged log-sum-exp rows the vote items need.
+    // Each walks its own kind of item in schedule order, so publishing never waits for
+    // another CTA and the fetcher runs as far ahead as its shared-memory buffers allow.
+    const bool publisher = warp == 2 + EPI_WARPS;
     int nstat = 0, nvote = 0;
     for_each_item(a, cta, G, /*lag=*/1, [&](const Item& it) {
+      if ((it.vote != 0) == publisher) return true;  // the other warp's kind of item
       if (!it.vote) {
         // merge the replicas and the two warpgroups (fixed order), publish, count
         const int pb = nstat % NPB;
