@@ -24,8 +24,11 @@
 //
 // Warp roles: warp 0 issues TMA loads (K tiles into a ring of stages, Q per work item
 // into two buffers), warp 1 issues tcgen05.mma into four TMEM accumulator buffers, warps
-// 2-9 (two warpgroups, alternating tiles) read the accumulators back with tcgen05.ld and
-// do the fp32 softmax arithmetic, warps 10 and 11 are the book-keepers: warp 10 merges and
+// 2-9 (two warpgroups) read the accumulators back with tcgen05.ld and do the fp32 softmax
+// arithmetic; with 64 or more query columns per unit a second set of eight softmax warps
+// (12-19) takes every other tile, each warpgroup of a set working on half of the columns:
+// the epilogue is bound by instruction latency, and four warps per scheduler hide it where
+// two do not.  Warps 10 and 11 are the book-keepers: warp 10 merges and
 // publishes the partial statistics the softmax warps leave in shared memory, warp 11
 // fetches the merged log-sum-exp of the coming vote items while the softmax warps are
 // still busy.  The single-thread roles (TMA and MMA issue) are entered through elect.sync:
@@ -47,8 +50,10 @@ constexpr int STAGES = 4;
 constexpr int NBUF = 4;               // TMEM accumulator buffers of 128 columns
 constexpr int TMEM_COLS = 512;
 constexpr int SUBTILE_BYTES = 128 * 128;  // 128 rows x 64 bf16, 128-byte swizzled
-constexpr int THREADS = 384;          // producer, MMA, 8 softmax warps, publisher, lse fetcher
-constexpr int EPI_WARPS = 8;
+constexpr int EPI_WARPS = 8;           // softmax warps per set (two warpgroups)
+// Warps: 0 producer, 1 MMA issuer, 2-9 softmax set 0, 10 publisher, 11 lse fetcher and, in
+// split mode, 12-19 softmax set 1.
+constexpr int threads_for(bool split) { return split ? 640 : 384; }
 #ifndef WAVE_MIB
 #define WAVE_MIB 64
 #endif
@@ -56,7 +61,7 @@ constexpr int EPI_WARPS = 8;
 #define WAVE_LAG 2
 #endif
 constexpr long long WAVE_BYTES = static_cast<long long>(WAVE_MIB) << 20;
-constexpr int NPB = 8;                // buffers for partial statistics (book-keeper queue)
+constexpr int NPB = 4;                // buffers for partial statistics (book-keeper queue)
 constexpr int NLB = 16;               // buffers for merged log-sum-exp rows
 
 struct ScoreArgs {
@@ -87,8 +92,8 @@ struct Smem {
   // pfull[NPB], pempty[NPB] (partial statistics), lfull[NLB], lempty[NLB] (log-sum-exp)
   static constexpr int NBAR = 2 * STAGES + 2 * NBUF + 5 + 2 * NPB + 2 * NLB;
   static constexpr int OFF_MISC = OFF_BAR + ((NBAR * 8 + 15) & ~15);  // tmem ptr, abort
-  static constexpr int OFF_PART = OFF_MISC + 16;              // float2 [NPB][8][32]
-  static constexpr int OFF_LSE = OFF_PART + NPB * 8 * 32 * 8; // float [NLB][128]
+  static constexpr int OFF_PART = OFF_MISC + 16;              // float2 [NPB][2 sets][8][32]
+  static constexpr int OFF_LSE = OFF_PART + NPB * 16 * 32 * 8; // float [NLB][128]
   static constexpr int TOTAL = OFF_LSE + NLB * 128 * 4;
   static_assert(OFF_PART % 16 == 0 && OFF_LSE % 16 == 0, "float4 reads of the lse buffers");
   static constexpr int DYN_BYTES = TOTAL + 1024;            // slack for 1024-byte alignment
@@ -183,15 +188,14 @@ __device__ __forceinline__ void for_each_item(const ScoreArgs& a, int cta, int G
 
 // NCH = npad / 32: how many 32-column chunks of the accumulator a thread reads per tile.
 template <int D, int NCH, bool SPLIT>
-// Split mode is built for 128 registers per thread (a launch bound of 512 threads): it has
-// no spills there and runs faster than with the 168 the thread count alone would allow.
-__global__ void __launch_bounds__(SPLIT ? 512 : THREADS, 1)
+__global__ void __launch_bounds__(threads_for(SPLIT), 1)
 score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
              const ScoreArgs a) {
   using SM = Smem<D>;
   constexpr int SUBT = SM::SUBT;
   constexpr int NPAD = NCH * 32;
   constexpr int REPS = 128 / NPAD;
+  constexpr int NSET = SPLIT ? 2 : 1;  // sets of softmax warps
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
@@ -240,12 +244,12 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       mbar_init(bar_qe(b), 1);
     }
     for (int b = 0; b < NPB; ++b) {
-      mbar_init(bar_pf(b), EPI_WARPS);
+      mbar_init(bar_pf(b), EPI_WARPS * NSET);
       mbar_init(bar_pe(b), 1);
     }
     for (int b = 0; b < NLB; ++b) {
       mbar_init(bar_lf(b), 1);
-      mbar_init(bar_le(b), EPI_WARPS);
+      mbar_init(bar_le(b), EPI_WARPS * NSET);
     }
     mbar_init(bar_drain, 1);
     *abort_s = 0;
@@ -377,14 +381,17 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         mbar_wait_drain(bar_drain, 0);
       }
     }
-  } else if (warp < 2 + EPI_WARPS) {
+  } else if (warp < 2 + EPI_WARPS || warp >= 4 + EPI_WARPS) {
     // ------------------------------------------------------------ softmax warps
     // SPLIT: both warpgroups work on every tile, each on half of the accumulator columns
     // (CPT columns per thread); the -lse values of a vote item then fit in registers.
     // Otherwise the warpgroups alternate tiles and take all NPAD columns.
     constexpr int CPT = SPLIT ? NPAD / 2 : NPAD;
     constexpr int VCH = CPT / 32;
-    const int wg = (warp - 2) >> 2;
+    // SPLIT also has two sets of softmax warps: set 0 takes the even tiles (by ring position)
+    // and set 1 the odd ones, so four warps per scheduler hide each other's latencies.
+    const int set = warp >= 4 + EPI_WARPS ? 1 : 0;
+    const int wg = ((set ? warp - (4 + EPI_WARPS) : warp - 2) >> 2);
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     const uint32_t lane_sel = static_cast<uint32_t>(32 * q) << 16;
     const int rrow = 32 * q + lane;  // TMEM lane
@@ -405,7 +412,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         float m2 = -INFINITY;  // running max, log2 domain
         float l = 0.f;         // running sum of exp2(x - m2)
         for (int k = 0; k < nt; ++k, ++git) {
-          if (!SPLIT && (git & 1) != wg) continue;
+          if ((git & 1) != (SPLIT ? set : wg)) continue;
           const int buf = git & (NBUF - 1);
           const uint32_t ub = (git / NBUF) & 1;
           if (!mbar_wait_warp(bar_tf(buf), ub, abort_s, WAIT_EPI_TMEM_FULL)) return false;
@@ -459,7 +466,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         const int pb = nstat % NPB;
         if (!mbar_wait_warp(bar_pe(pb), ((nstat / NPB) & 1) ^ 1, abort_s, WAIT_PART_EMPTY))
           return false;
-        part_s[(pb * 8 + wg * 4 + q) * 32 + lane] = make_float2(m2, l);
+        part_s[((pb * 2 + set) * 8 + wg * 4 + q) * 32 + lane] = make_float2(m2, l);
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_pf(pb));
         ++nstat;
@@ -469,21 +476,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       const int lb = nvote % NLB;
       if (!mbar_wait_warp(bar_lf(lb), (nvote / NLB) & 1, abort_s, WAIT_LSE_FULL)) return false;
       const float* lse_b = lse_s + lb * MAX_COLS;
-      float lse_r[SPLIT ? VCH : 1][32];  // -lse of this thread's columns (SPLIT only)
-      if (SPLIT) {
-#pragma unroll
-        for (int ch = 0; ch < VCH; ++ch)
-#pragma unroll
-          for (int c4 = 0; c4 < 8; ++c4) {
-            const float4 z = *reinterpret_cast<const float4*>(lse_b + coff + ch * 32 + c4 * 4);
-            lse_r[ch][c4 * 4 + 0] = z.x;
-            lse_r[ch][c4 * 4 + 1] = z.y;
-            lse_r[ch][c4 * 4 + 2] = z.z;
-            lse_r[ch][c4 * 4 + 3] = z.w;
-          }
-      }
       for (int k = 0; k < nt; ++k, ++git) {
-        if (!SPLIT && (git & 1) != wg) continue;
+        if ((git & 1) != (SPLIT ? set : wg)) continue;
         const int buf = git & (NBUF - 1);
         const uint32_t ub = (git / NBUF) & 1;
         if (!mbar_wait_warp(bar_tf(buf), ub, abort_s, WAIT_EPI_TMEM_FULL)) return false;
@@ -518,13 +512,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
               float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
               for (int t4 = 0; t4 < 4; ++t4) {
-                float4 z;
-                if (SPLIT) {
-                  z = make_float4(lse_r[ch][hf * 16 + 4 * t4 + 0], lse_r[ch][hf * 16 + 4 * t4 + 1],
-                                  lse_r[ch][hf * 16 + 4 * t4 + 2], lse_r[ch][hf * 16 + 4 * t4 + 3]);
-                } else {
-                  z = *reinterpret_cast<const float4*>(lse_b + ch * 32 + hf * 16 + 4 * t4);
-                }
+                // -lse of four adjacent columns: one broadcast read for the whole warp
+                const float4 z =
+                    *reinterpret_cast<const float4*>(lse_b + coff + ch * 32 + hf * 16 + 4 * t4);
                 a0 += ex2_approx(fmaf(vc[hf * 16 + 4 * t4 + 0], a.c2, z.x));
                 a1 += ex2_approx(fmaf(vc[hf * 16 + 4 * t4 + 1], a.c2, z.y));
                 a2 += ex2_approx(fmaf(vc[hf * 16 + 4 * t4 + 2], a.c2, z.z));
@@ -576,7 +566,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     // last to publish); warp 11 fetches the merged log-sum-exp rows the vote items need.
     // Each walks its own kind of item in schedule order, so publishing never waits for
     // another CTA and the fetcher runs as far ahead as its shared-memory buffers allow.
-    const bool publisher = warp == 2 + EPI_WARPS;
+    const bool publisher = warp == 2 + EPI_WARPS;  // warp 10; warp 11 is the fetcher
     int nstat = 0, nvote = 0;
     for_each_item(a, cta, G, /*lag=*/1, [&](const Item& it) {
       if ((it.vote != 0) == publisher) return true;  // the other warp's kind of item
@@ -585,16 +575,17 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         const int pb = nstat % NPB;
         if (!mbar_wait_warp_relaxed(bar_pf(pb), (nstat / NPB) & 1, abort_s, WAIT_PART_FULL))
           return false;
-        const float2* ps = part_s + pb * 8 * 32;
+        const float2* ps = part_s + pb * 16 * 32;
         for (int c = lane; c < a.ncols; c += 32) {
           float M = -INFINITY;
-          for (int w2 = 0; w2 < 2; ++w2)
+          for (int w2 = 0; w2 < 2 * NSET; ++w2)
             for (int r = 0; r < REPS; ++r) {
               const int row = r * NPAD + c;
               M = fmaxf(M, ps[(w2 * 4 + (row >> 5)) * 32 + (row & 31)].x);
             }
+          M = fmaxf(M, -1e30f);
           float S = 0.f;
-          for (int w2 = 0; w2 < 2; ++w2)
+          for (int w2 = 0; w2 < 2 * NSET; ++w2)
             for (int r = 0; r < REPS; ++r) {
               const int row = r * NPAD + c;
               const float2 p = ps[(w2 * 4 + (row >> 5)) * 32 + (row & 31)];
@@ -759,7 +750,7 @@ cudaError_t run_scores(const CUtensorMap& tmK, const CUtensorMap& tmQ, const Sco
   // than the SM count: every CTA becomes resident as soon as the stream's earlier work
   // has drained, so a CTA that waits for another CTA's partial statistics is waiting for
   // a CTA that runs.  The waits are bounded in any case.
-  score_kernel<D, NCH, SPLIT><<<dim3(grid), dim3(THREADS), Smem<D>::DYN_BYTES, stream>>>(tmK, tmQ, a);
+  score_kernel<D, NCH, SPLIT><<<dim3(grid), dim3(threads_for(SPLIT)), Smem<D>::DYN_BYTES, stream>>>(tmK, tmQ, a);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   *launches += 1;
