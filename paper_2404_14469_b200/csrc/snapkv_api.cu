@@ -19,7 +19,7 @@ WorkspaceLayout make_layout(const ScorePlan& p, int B, int Hq, int n, bool need_
   w.off_counters = off;
   off = align_up(off + sizeof(int) * static_cast<size_t>(p.units), 256);
   w.off_partials = off;
-  off = align_up(off + sizeof(float2) * static_cast<size_t>(p.units) * p.maxseg * MAX_COLS, 256);
+  off = align_up(off + sizeof(float) * static_cast<size_t>(p.units) * p.maxseg * MAX_COLS, 256);
   w.off_lse = off;
   off = align_up(off + sizeof(float) * static_cast<size_t>(p.units) * MAX_COLS, 256);
   w.off_vote = off;
@@ -112,7 +112,7 @@ snapkv_status_t snapkv_window_scores(const void* q_obs, const void* k, int B, in
   int launches = 0;
   cudaError_t e = launch_window_scores(
       q_obs, k, B, Hq, Hkv, L, d, W, p, out_vote, reinterpret_cast<int*>(ws + w.off_status),
-      reinterpret_cast<int*>(ws + w.off_counters), reinterpret_cast<float2*>(ws + w.off_partials),
+      reinterpret_cast<int*>(ws + w.off_counters), reinterpret_cast<float*>(ws + w.off_partials),
       reinterpret_cast<float*>(ws + w.off_lse), s, &launches);
   if (e != cudaSuccess) return SNAPKV_ERR_CUDA;
   g_last_launches = launches;
@@ -192,7 +192,7 @@ snapkv_status_t snapkv_compress(const void* q_obs, const void* k, const void* v,
   if (launch_window_scores(q_obs, k, B, Hq, Hkv, L, d, W, p, vote,
                            reinterpret_cast<int*>(ws + w.off_status),
                            reinterpret_cast<int*>(ws + w.off_counters),
-                           reinterpret_cast<float2*>(ws + w.off_partials),
+                           reinterpret_cast<float*>(ws + w.off_partials),
                            reinterpret_cast<float*>(ws + w.off_lse), s, &launches) != cudaSuccess)
     return SNAPKV_ERR_CUDA;
   if (launch_pool_topk(vote, B * Hq, n, pool_kernel, pool_type, ksel, out_idx,

@@ -26,6 +26,7 @@ enum WaitCode {
   WAIT_PART_FULL = 9,
   WAIT_LSE_FULL = 10,
   WAIT_LSE_EMPTY = 11,
+  WAIT_MERGE_COPY = 12,
 };
 
 // How the scoring passes split the work.  A "unit" is one (batch, KV head, head
@@ -59,7 +60,7 @@ size_t select_scratch_bytes(int rows, int n);  // 0 when the rows fit one CTA
 // kernel starts (the callers clear it together with the status block).
 cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv, int L,
                                  int d, int W, const ScorePlan& plan, float* vote, int* status,
-                                 int* counters, float2* partials, float* lse2, cudaStream_t stream,
+                                 int* counters, float* partials, float* lse2, cudaStream_t stream,
                                  int* launches);
 
 // Pool + top-k over `rows` rows of fp32 votes.  `pooled_scratch` (select_scratch_bytes bytes)

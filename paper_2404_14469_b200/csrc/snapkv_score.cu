@@ -61,8 +61,9 @@ constexpr int threads_for(bool split) { return split ? 640 : 384; }
 #define WAVE_LAG 2
 #endif
 constexpr long long WAVE_BYTES = static_cast<long long>(WAVE_MIB) << 20;
-constexpr int NPB = 4;                // buffers for partial statistics (book-keeper queue)
-constexpr int NLB = 16;               // buffers for merged log-sum-exp rows
+constexpr int NPB = 2;                // buffers for partial statistics (book-keeper queue)
+constexpr int NLB = 8;                // buffers for merged log-sum-exp rows
+constexpr int MERGE_SEGS = 32;        // partials staged in shared memory per merge round
 
 struct ScoreArgs {
   int L, n, W;
@@ -73,7 +74,7 @@ struct ScoreArgs {
   int maxseg;               // partial slots per unit
   int pipelined;            // how many waves the statistics run ahead of the votes (>= 1)
   float c2;                 // log2(e) / sqrt(d)
-  float2* partials;         // [units][maxseg][MAX_COLS] (max, sum) in the log2 domain
+  float* partials;          // [units][maxseg][MAX_COLS] log2-sum-exp of one CTA's share
   float* lse2;              // [units][MAX_COLS] minus the merged log2-sum-exp per window row
   int* counters;            // [units] published partials (+1 once lse2 is written)
   int* status;
@@ -89,13 +90,16 @@ struct Smem {
   static constexpr int OFF_K = 2 * Q_BYTES;
   static constexpr int OFF_BAR = OFF_K + STAGES * STAGE_BYTES;
   // barriers: full[STAGES], empty[STAGES], tf[NBUF], te[NBUF], qfull[2], qempty[2], drain,
-  // pfull[NPB], pempty[NPB] (partial statistics), lfull[NLB], lempty[NLB] (log-sum-exp)
-  static constexpr int NBAR = 2 * STAGES + 2 * NBUF + 5 + 2 * NPB + 2 * NLB;
+  // pfull[NPB], pempty[NPB] (partial statistics), lfull[NLB], lempty[NLB] (log-sum-exp),
+  // merge (bulk copy of a unit's partials)
+  static constexpr int NBAR = 2 * STAGES + 2 * NBUF + 5 + 2 * NPB + 2 * NLB + 1;
   static constexpr int OFF_MISC = OFF_BAR + ((NBAR * 8 + 15) & ~15);  // tmem ptr, abort
   static constexpr int OFF_PART = OFF_MISC + 16;              // float2 [NPB][2 sets][8][32]
   static constexpr int OFF_LSE = OFF_PART + NPB * 16 * 32 * 8; // float [NLB][128]
-  static constexpr int TOTAL = OFF_LSE + NLB * 128 * 4;
-  static_assert(OFF_PART % 16 == 0 && OFF_LSE % 16 == 0, "float4 reads of the lse buffers");
+  static constexpr int OFF_MERGE = OFF_LSE + NLB * 128 * 4;   // float [MERGE_SEGS][128]
+  static constexpr int TOTAL = OFF_MERGE + MERGE_SEGS * 128 * 4;
+  static_assert(OFF_PART % 16 == 0 && OFF_LSE % 16 == 0 && OFF_MERGE % 16 == 0,
+                "float4 reads of the lse buffers, bulk copies into the merge buffer");
   static constexpr int DYN_BYTES = TOTAL + 1024;            // slack for 1024-byte alignment
 };
 
@@ -220,6 +224,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
   auto bar_pe = [&](int b) { return bar0 + 8u * (BAR_P + NPB + b); };
   auto bar_lf = [&](int b) { return bar0 + 8u * (BAR_P + 2 * NPB + b); };
   auto bar_le = [&](int b) { return bar0 + 8u * (BAR_P + 2 * NPB + NLB + b); };
+  const uint32_t bar_merge = bar0 + 8u * (BAR_P + 2 * NPB + 2 * NLB);
   volatile uint32_t* tmem_ptr_s = reinterpret_cast<volatile uint32_t*>(smem + SM::OFF_MISC);
   volatile int* abort_s = reinterpret_cast<volatile int*>(smem + SM::OFF_MISC + 4);
   float2* part_s = reinterpret_cast<float2*>(smem + SM::OFF_PART);
@@ -252,6 +257,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       mbar_init(bar_le(b), EPI_WARPS * NSET);
     }
     mbar_init(bar_drain, 1);
+    mbar_init(bar_merge, 1);
     *abort_s = 0;
     mbar_fence_init();
   }
@@ -279,6 +285,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     if (elect_one()) {
       tma_prefetch_desc(&tmK);
       tma_prefetch_desc(&tmQ);
+      const uint64_t pol_first = l2_policy_evict_first();
       int git = 0;      // tiles issued so far (ring position)
       int nitem = 0;    // items started so far (Q buffer position)
       for_each_item(a, cta, G, a.pipelined, [&](const Item& it) {
@@ -305,9 +312,14 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           if (!mbar_wait_thread(bar_empty(s), ph ^ 1, abort_s, WAIT_PRODUCER_EMPTY)) return false;
           mbar_expect_tx(bar_full(s), SM::STAGE_BYTES);
           const int key0 = tile_of(it, k) * TILE_KEYS;
-          for (int sb = 0; sb < SUBT; ++sb)
-            tma_load_3d(stage_addr(s, sb), &tmK, bar_full(s), sb * 64,
-                        key0, ukv);
+          // the vote pass is the last reader of a key tile: its lines may leave L2 first,
+          // which keeps the next wave's statistics-pass lines resident instead
+          for (int sb = 0; sb < SUBT; ++sb) {
+            if (it.vote)
+              tma_load_3d_hint(stage_addr(s, sb), &tmK, bar_full(s), sb * 64, key0, ukv, pol_first);
+            else
+              tma_load_3d(stage_addr(s, sb), &tmK, bar_full(s), sb * 64, key0, ukv);
+          }
         }
         return true;
       });
@@ -567,7 +579,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     // Each walks its own kind of item in schedule order, so publishing never waits for
     // another CTA and the fetcher runs as far ahead as its shared-memory buffers allow.
     const bool publisher = warp == 2 + EPI_WARPS;  // warp 10; warp 11 is the fetcher
-    int nstat = 0, nvote = 0;
+    int nstat = 0, nvote = 0, nmerge = 0;
+    const float* merge_s = reinterpret_cast<const float*>(smem + SM::OFF_MERGE);
     for_each_item(a, cta, G, /*lag=*/1, [&](const Item& it) {
       if ((it.vote != 0) == publisher) return true;  // the other warp's kind of item
       if (!it.vote) {
@@ -591,8 +604,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
               const float2 p = ps[(w2 * 4 + (row >> 5)) * 32 + (row & 31)];
               S += p.y * ex2_approx(p.x - M);
             }
+          // log2 of this CTA's share of the row's softmax normaliser (-inf if it saw no key)
           a.partials[(static_cast<size_t>(it.unit) * a.maxseg + it.slot) * MAX_COLS + c] =
-              make_float2(M, S);
+              M + log2f(S);
         }
         __threadfence();
         __syncwarp();
@@ -603,37 +617,43 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         }
         if (__shfl_sync(0xffffffffu, last, 0)) {
           // this was the unit's last partial: fold all of them, in slot order, into one
-          // -log2-sum-exp per window row, then raise the count once more to say so.
-          // Each lane owns four adjacent window rows; loads go eight segments at a time.
+          // -log2-sum-exp per window row, then raise the count once more to say so.  The
+          // unit's partials are contiguous: one bulk copy brings up to MERGE_SEGS of them
+          // into shared memory (a single trip through the loaded memory system instead of
+          // one per batch of register loads); each lane then owns four adjacent rows.
           (void)ld_acquire(a.counters + it.unit);
+          fence_proxy_async();
+          const float* pp = a.partials + static_cast<size_t>(it.unit) * a.maxseg * MAX_COLS;
           const int c4 = lane * 4;
-          if (c4 < a.ncols) {
-            const float4* pp = reinterpret_cast<const float4*>(
-                a.partials + static_cast<size_t>(it.unit) * a.maxseg * MAX_COLS + c4);
-            float M[4], S[4];
+          float M[4], S[4];
 #pragma unroll
-            for (int t = 0; t < 4; ++t) { M[t] = -INFINITY; S[t] = 0.f; }
-            for (int s0 = 0; s0 < it.nseg; s0 += 8) {
-              float4 x[8][2];
-#pragma unroll
-              for (int uu = 0; uu < 8; ++uu)
-                if (s0 + uu < it.nseg) {
-                  x[uu][0] = __ldcg(pp + static_cast<size_t>(s0 + uu) * (MAX_COLS / 2));
-                  x[uu][1] = __ldcg(pp + static_cast<size_t>(s0 + uu) * (MAX_COLS / 2) + 1);
-                }
-#pragma unroll
-              for (int uu = 0; uu < 8; ++uu)
-                if (s0 + uu < it.nseg) {
-                  const float m[4] = {x[uu][0].x, x[uu][0].z, x[uu][1].x, x[uu][1].z};
-                  const float sv[4] = {x[uu][0].y, x[uu][0].w, x[uu][1].y, x[uu][1].w};
-#pragma unroll
-                  for (int t = 0; t < 4; ++t) {
-                    const float Mn = fmaxf(M[t], m[t]);
-                    S[t] = S[t] * ex2_approx(M[t] - Mn) + sv[t] * ex2_approx(m[t] - Mn);
-                    M[t] = Mn;
-                  }
-                }
+          for (int t = 0; t < 4; ++t) { M[t] = -INFINITY; S[t] = 0.f; }
+          for (int s0 = 0; s0 < it.nseg; s0 += MERGE_SEGS, ++nmerge) {
+            const int ns = min(MERGE_SEGS, it.nseg - s0);
+            if (lane == 0) {
+              mbar_expect_tx(bar_merge, ns * MAX_COLS * 4);
+              bulk_load(sbase + SM::OFF_MERGE, pp + static_cast<size_t>(s0) * MAX_COLS,
+                        ns * MAX_COLS * 4, bar_merge);
             }
+            if (!mbar_wait_warp_relaxed(bar_merge, nmerge & 1, abort_s, WAIT_MERGE_COPY)) {
+              mbar_wait_drain(bar_merge, nmerge & 1);  // never leave with the copy in flight
+              return false;
+            }
+            if (c4 < a.ncols) {
+              for (int sg = 0; sg < ns; ++sg) {
+                const float4 x = *reinterpret_cast<const float4*>(merge_s + sg * MAX_COLS + c4);
+                const float pv[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                  const float Mn = fmaxf(fmaxf(M[t], pv[t]), -1e30f);
+                  S[t] = S[t] * ex2_approx(M[t] - Mn) + ex2_approx(pv[t] - Mn);
+                  M[t] = Mn;
+                }
+              }
+            }
+            __syncwarp();  // all lanes are done with the buffer before the next copy lands
+          }
+          if (c4 < a.ncols) {
             float4 out;
             out.x = -(M[0] + log2f(S[0]));
             out.y = -(M[1] + log2f(S[1]));
@@ -811,7 +831,7 @@ bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* pla
 
 cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv, int L,
                                  int d, int W, const ScorePlan& plan, float* vote, int* status,
-                                 int* counters, float2* partials, float* lse2, cudaStream_t stream,
+                                 int* counters, float* partials, float* lse2, cudaStream_t stream,
                                  int* launches) {
   CUtensorMap tmK, tmQ;
   {
