@@ -187,7 +187,9 @@ __device__ __forceinline__ int key_slot(int j) { return j + (j >> 5); }
 constexpr int CAND_CAP = 2048;   // keys of the first-pass bin that are refined from a list
 constexpr int MASK_WORDS = 2;    // a thread owns at most 64 positions (SEL_SMEM_KEYS / SEL_THREADS = 48)
 
-template <int RMAX>
+// PT = -1: pooling radius r <= RMAX and pool type are run-time values.  PT = 0 (max) or 1
+// (avg): the radius is exactly RMAX, so the window loop has no per-element tests.
+template <int RMAX, int PT>
 __global__ void __launch_bounds__(SEL_THREADS, 1)
 pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_type, int ept,
                       int ksel, int32_t* __restrict__ out_idx) {
@@ -243,7 +245,8 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
 #pragma unroll
         for (int t = 0; t <= 2 * RMAX; ++t) {
           const int off = t - RMAX;
-          if (off >= -r && off <= r) p = (pool_type == 0) ? fmaxf(p, w[i + t]) : p + w[i + t];
+          if (PT >= 0 || (off >= -r && off <= r))
+            p = ((PT >= 0) ? (PT == 0) : (pool_type == 0)) ? fmaxf(p, w[i + t]) : p + w[i + t];
         }
         const int j = base + sb + i;
         uint32_t key = 0u;  // positions past the row end rank below every real key
@@ -680,24 +683,31 @@ cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel
     cudaError_t e = cudaFuncSetAttribute(pool_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          SEL_SMEM_KEYS * 4);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(pool_topk_fast_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             FAST_SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(pool_topk_fast_kernel<7>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             FAST_SMEM_BYTES);
-    if (e != cudaSuccess) return e;
+#define SNAPKV_FAST_ATTR(RM, P)                                                              \
+  e = cudaFuncSetAttribute(pool_topk_fast_kernel<RM, P>,                                     \
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, FAST_SMEM_BYTES);    \
+  if (e != cudaSuccess) return e;
+    SNAPKV_FAST_ATTR(3, -1) SNAPKV_FAST_ATTR(7, -1)
+    SNAPKV_FAST_ATTR(2, 0) SNAPKV_FAST_ATTR(2, 1) SNAPKV_FAST_ATTR(3, 0) SNAPKV_FAST_ATTR(3, 1)
+    SNAPKV_FAST_ATTR(6, 0) SNAPKV_FAST_ATTR(6, 1)
+#undef SNAPKV_FAST_ATTR
     attr_done = true;
   }
   const int r = pool_kernel >> 1;
   if (n <= SEL_SMEM_KEYS && r <= 7) {
     const int ept = (((n + SEL_THREADS - 1) / SEL_THREADS) + 7) & ~7;
     const int words = key_slot_host(SEL_THREADS * ept) + 1;
-    if (r <= 3)
-      pool_topk_fast_kernel<3><<<rows, SEL_THREADS, words * 4, stream>>>(vote, n, r, pool_type, ept,
-                                                                       ksel, out_idx);
-    else
-      pool_topk_fast_kernel<7><<<rows, SEL_THREADS, words * 4, stream>>>(vote, n, r, pool_type, ept,
-                                                                       ksel, out_idx);
+#define SNAPKV_FAST_LAUNCH(RM, P)                                                            \
+  pool_topk_fast_kernel<RM, P><<<rows, SEL_THREADS, words * 4, stream>>>(vote, n, r, pool_type, \
+                                                                        ept, ksel, out_idx)
+    // the paper's kernel sizes 5, 7 and 13 have instantiations of their own
+    const bool mx = pool_type == 0;
+    if (r == 2) { if (mx) SNAPKV_FAST_LAUNCH(2, 0); else SNAPKV_FAST_LAUNCH(2, 1); }
+    else if (r == 3) { if (mx) SNAPKV_FAST_LAUNCH(3, 0); else SNAPKV_FAST_LAUNCH(3, 1); }
+    else if (r == 6) { if (mx) SNAPKV_FAST_LAUNCH(6, 0); else SNAPKV_FAST_LAUNCH(6, 1); }
+    else if (r <= 3) SNAPKV_FAST_LAUNCH(3, -1);
+    else SNAPKV_FAST_LAUNCH(7, -1);
+#undef SNAPKV_FAST_LAUNCH
     *launches += 1;
     return cudaGetLastError();
   }
