@@ -4,11 +4,28 @@
 #include <stdint.h>
 
 #include "../../include/snapkv.h"
+#include "launch.cuh"
 #include "snapkv_internal.h"
 
 namespace snapkv {
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Clears the status block and the unit counters behind it (a multiple of 256 bytes).  A
+// kernel rather than a memset so that the scoring kernel behind it can be made resident early.
+__global__ void clear_kernel(uint4* p, int n16) {
+  pdl_launch_dependents();
+  pdl_wait();
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += gridDim.x * blockDim.x)
+    p[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+static cudaError_t launch_clear(uint8_t* ws, const WorkspaceLayout& w, cudaStream_t s) {
+  const int n16 = static_cast<int>((w.off_partials - w.off_status) / 16);
+  const int blocks = n16 > 256 * 64 ? 64 : (n16 + 255) / 256;
+  return launch_pdl(clear_kernel, dim3(blocks), dim3(256), 0, s,
+                    reinterpret_cast<uint4*>(ws + w.off_status), n16);
+}
 
 WorkspaceLayout make_layout(const ScorePlan& p, int B, int Hq, int n, bool need_vote,
                             bool need_pooled) {
@@ -106,10 +123,8 @@ snapkv_status_t snapkv_window_scores(const void* q_obs, const void* k, int B, in
     return SNAPKV_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  // one memset clears the status block and the unit counters behind it
-  if (cudaMemsetAsync(ws + w.off_status, 0, w.off_partials - w.off_status, s) != cudaSuccess)
-    return SNAPKV_ERR_CUDA;
-  int launches = 0;
+  if (launch_clear(ws, w, s) != cudaSuccess) return SNAPKV_ERR_CUDA;
+  int launches = 1;
   cudaError_t e = launch_window_scores(
       q_obs, k, B, Hq, Hkv, L, d, W, p, out_vote, reinterpret_cast<int*>(ws + w.off_status),
       reinterpret_cast<int*>(ws + w.off_counters), reinterpret_cast<float*>(ws + w.off_partials),
@@ -184,9 +199,8 @@ snapkv_status_t snapkv_compress(const void* q_obs, const void* k, const void* v,
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < w.total)
     return SNAPKV_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  // one memset clears the status block and the unit counters behind it
-  if (cudaMemsetAsync(ws + w.off_status, 0, w.off_partials - w.off_status, s) != cudaSuccess)
-    return SNAPKV_ERR_CUDA;
+  if (launch_clear(ws, w, s) != cudaSuccess) return SNAPKV_ERR_CUDA;
+  launches += 1;
   float* vote = reinterpret_cast<float*>(ws + w.off_vote);
   const int ksel = budget - W;
   if (launch_window_scores(q_obs, k, B, Hq, Hkv, L, d, W, p, vote,

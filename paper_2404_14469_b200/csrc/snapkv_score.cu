@@ -39,6 +39,7 @@
 #include <math.h>
 #include <stdint.h>
 
+#include "launch.cuh"
 #include "sm100_ptx.cuh"
 #include "snapkv_internal.h"
 
@@ -195,6 +196,7 @@ template <int D, int NCH, bool SPLIT>
 __global__ void __launch_bounds__(threads_for(SPLIT), 1)
 score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
              const ScoreArgs a) {
+  pdl_launch_dependents();
   using SM = Smem<D>;
   constexpr int SUBT = SM::SUBT;
   constexpr int NPAD = NCH * 32;
@@ -265,6 +267,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_ptr_s)), TMEM_COLS);
     tmem_relinquish();
   }
+  // everything above touched only this CTA's shared memory and TMEM; from here on the
+  // kernel reads and writes global memory, so the previous kernel must be complete
+  pdl_wait();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -770,8 +775,10 @@ cudaError_t run_scores(const CUtensorMap& tmK, const CUtensorMap& tmQ, const Sco
   // than the SM count: every CTA becomes resident as soon as the stream's earlier work
   // has drained, so a CTA that waits for another CTA's partial statistics is waiting for
   // a CTA that runs.  The waits are bounded in any case.
-  score_kernel<D, NCH, SPLIT><<<dim3(grid), dim3(threads_for(SPLIT)), Smem<D>::DYN_BYTES, stream>>>(tmK, tmQ, a);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = launch_pdl(score_kernel<D, NCH, SPLIT>, dim3(grid), dim3(threads_for(SPLIT)),
+                             Smem<D>::DYN_BYTES, stream, tmK, tmQ, a);
+  if (e != cudaSuccess) return e;
+  e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   *launches += 1;
   return cudaSuccess;
