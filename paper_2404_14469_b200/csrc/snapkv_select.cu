@@ -184,6 +184,14 @@ pool_topk_kernel(const float* __restrict__ vote, int n, int pool_kernel, int poo
 // bank conflicts.  The first histogram pass bins (key - min) >> shift with the shift
 // chosen from the row's key range, so the bins are spread over the values that occur.
 __device__ __forceinline__ int key_slot(int j) { return j + (j >> 5); }
+// Layout of the one-CTA-per-row kernel: four pad words after every 32 keys.  A thread's run
+// starts at a multiple of 8 keys, so it reads and writes its keys four at a time as aligned
+// 16-byte vectors, and the runs of eight neighbouring threads fall into different banks.
+__device__ __forceinline__ int key_slot4(int j) { return j + ((j >> 5) << 2); }
+__device__ __forceinline__ uint4 ld_keys4(const uint32_t* keys, int j) {
+  return *reinterpret_cast<const uint4*>(keys + key_slot4(j));
+}
+constexpr int FAST_MAX_KEYS = 40960;  // 40 keys per thread: what fits with the padding
 constexpr int CAND_CAP = 2048;   // keys of the first-pass bin that are refined from a list
 constexpr int MASK_WORDS = 2;    // a thread owns at most 64 positions (SEL_SMEM_KEYS / SEL_THREADS = 48)
 
@@ -193,7 +201,7 @@ template <int RMAX, int PT>
 __global__ void __launch_bounds__(SEL_THREADS, 1)
 pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_type, int ept,
                       int ksel, int32_t* __restrict__ out_idx) {
-  extern __shared__ uint32_t keys[];
+  extern __shared__ __align__(16) uint32_t keys[];
   __shared__ int hist[NBINS];
   __shared__ int warp_sums[SEL_WARPS];
   __shared__ int scan_total;
@@ -215,30 +223,38 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
   {
     const int total = SEL_THREADS * ept;
     for (int j = threadIdx.x; j < total; j += SEL_THREADS)
-      keys[key_slot(j)] = (j < n) ? __float_as_uint(__ldg(vrow + j)) : 0u;
+      keys[key_slot4(j)] = (j < n) ? __float_as_uint(__ldg(vrow + j)) : 0u;
     __syncthreads();
-    float w[2 * RMAX + 8];
+    // a[]: the last RMAX values before the current block of 8, the block, the next block
+    float a[RMAX + 16];
     float halo_r[RMAX > 0 ? RMAX : 1];
 #pragma unroll
     for (int i = 0; i < RMAX; ++i) {
       const int jl = base - RMAX + i;             // left neighbours
-      w[i] = (jl >= 0) ? __uint_as_float(keys[key_slot(jl)]) : 0.f;
+      a[i] = (jl >= 0) ? __uint_as_float(keys[key_slot4(jl)]) : 0.f;
       const int jr = base + ept + i;              // right neighbours
-      halo_r[i] = (jr < total) ? __uint_as_float(keys[key_slot(jr)]) : 0.f;
+      halo_r[i] = (jr < total) ? __uint_as_float(keys[key_slot4(jr)]) : 0.f;
     }
+    auto load8 = [&](int pos, float* dst) {       // own positions pos .. pos + 7
+      const uint4 x = ld_keys4(keys, pos), y = ld_keys4(keys, pos + 4);
+      dst[0] = __uint_as_float(x.x); dst[1] = __uint_as_float(x.y);
+      dst[2] = __uint_as_float(x.z); dst[3] = __uint_as_float(x.w);
+      dst[4] = __uint_as_float(y.x); dst[5] = __uint_as_float(y.y);
+      dst[6] = __uint_as_float(y.z); dst[7] = __uint_as_float(y.w);
+    };
+    auto next8 = [&](int sb_next, float* dst) {   // the block after sb_next - 8, or the halo
+      if (sb_next < ept) {
+        load8(base + sb_next, dst);
+      } else {
 #pragma unroll
-    for (int i = 0; i < RMAX; ++i) w[RMAX + i] = __uint_as_float(keys[key_slot(base + i)]);
-    __syncthreads();
-    for (int sb = 0; sb < ept; sb += 8) {
-      const bool last = (sb + 8 == ept);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        // position base + sb + RMAX + i: own (not yet overwritten) or a saved right neighbour
-        float x;
-        if (i >= 8 - RMAX && last) x = halo_r[(i >= 8 - RMAX) ? i - (8 - RMAX) : 0];
-        else x = __uint_as_float(keys[key_slot(base + sb + RMAX + i)]);
-        w[2 * RMAX + i] = x;
+        for (int i = 0; i < 8; ++i) dst[i] = (i < RMAX) ? halo_r[i < RMAX ? i : 0] : 0.f;
       }
+    };
+    load8(base, a + RMAX);
+    __syncthreads();  // every neighbour value is in registers before anybody overwrites
+    next8(8, a + RMAX + 8);
+    for (int sb = 0; sb < ept; sb += 8) {
+      uint32_t out[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         float p = 0.f;  // votes are >= 0: zero is neutral for max and is the avg padding
@@ -246,7 +262,7 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
         for (int t = 0; t <= 2 * RMAX; ++t) {
           const int off = t - RMAX;
           if (PT >= 0 || (off >= -r && off <= r))
-            p = ((PT >= 0) ? (PT == 0) : (pool_type == 0)) ? fmaxf(p, w[i + t]) : p + w[i + t];
+            p = ((PT >= 0) ? (PT == 0) : (pool_type == 0)) ? fmaxf(p, a[i + t]) : p + a[i + t];
         }
         const int j = base + sb + i;
         uint32_t key = 0u;  // positions past the row end rank below every real key
@@ -255,10 +271,15 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
           kmin = min(kmin, key);
           kmax = max(kmax, key);
         }
-        keys[key_slot(j)] = key;
+        out[i] = key;
       }
 #pragma unroll
-      for (int i = 0; i < 2 * RMAX; ++i) w[i] = w[i + 8];
+      for (int i = 0; i < RMAX + 8; ++i) a[i] = a[i + 8];
+      // the block after the next one is still untouched; the current one is done with
+      next8(sb + 16, a + RMAX + 8);
+      *reinterpret_cast<uint4*>(keys + key_slot4(base + sb)) = make_uint4(out[0], out[1], out[2], out[3]);
+      *reinterpret_cast<uint4*>(keys + key_slot4(base + sb + 4)) =
+          make_uint4(out[4], out[5], out[6], out[7]);
     }
   }
   kmin = __reduce_min_sync(0xffffffffu, kmin);
@@ -297,17 +318,22 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
       __syncthreads();
       if (!use_list) {
         int cur = -1, cnt = 0;
-        for (int i = 0; i < ept; ++i) {
-          const uint32_t key = keys[key_slot(base + i)];
-          const uint32_t rel = key - lo;
-          if (key >= lo && rel <= width_m1) {
-            const int b = static_cast<int>(rel >> shift);
-            if (b != cur) {
-              if (cnt) atomicAdd(&hist[cur], cnt);
-              cur = b;
-              cnt = 0;
+        for (int i0 = 0; i0 < ept; i0 += 4) {
+          const uint4 kv = ld_keys4(keys, base + i0);
+          const uint32_t k4[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const uint32_t key = k4[u];
+            const uint32_t rel = key - lo;
+            if (key >= lo && rel <= width_m1) {
+              const int b = static_cast<int>(rel >> shift);
+              if (b != cur) {
+                if (cnt) atomicAdd(&hist[cur], cnt);
+                cur = b;
+                cnt = 0;
+              }
+              ++cnt;
             }
-            ++cnt;
           }
         }
         if (cnt) atomicAdd(&hist[cur], cnt);
@@ -344,13 +370,22 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
         first = false;
         const uint32_t hi_m1 = done ? 0u : ((1u << shift) - 1u);
         use_list = !done && in_bin <= CAND_CAP;
-        for (int i = 0; i < ept; ++i) {
-          const uint32_t key = keys[key_slot(base + i)];
-          const bool inb = key >= lo && key - lo <= hi_m1;
-          const bool gt = key >= lo && key - lo > hi_m1;
-          m_gt[i >> 5] |= static_cast<uint32_t>(gt) << (i & 31);
-          m_in[i >> 5] |= static_cast<uint32_t>(inb) << (i & 31);
-          if (inb && use_list) cand[atomicAdd(&ncand_s, 1)] = key;
+        for (int i0 = 0; i0 < ept; i0 += 4) {
+          const uint4 kv = ld_keys4(keys, base + i0);
+          const uint32_t k4[4] = {kv.x, kv.y, kv.z, kv.w};
+          uint32_t bg = 0u, bi = 0u;  // four bits each
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const uint32_t key = k4[u];
+            const bool inb = key >= lo && key - lo <= hi_m1;
+            const bool gt = key >= lo && key - lo > hi_m1;
+            bg |= static_cast<uint32_t>(gt) << u;
+            bi |= static_cast<uint32_t>(inb) << u;
+            if (inb && use_list) cand[atomicAdd(&ncand_s, 1)] = key;
+          }
+          // i0 is a multiple of 4: the four bits never straddle a mask word
+          if (i0 < 32) { m_gt[0] |= bg << i0; m_in[0] |= bi << i0; }
+          else { m_gt[1] |= bg << (i0 - 32); m_in[1] |= bi << (i0 - 32); }
         }
         __syncthreads();
         ncand = ncand_s;
@@ -381,7 +416,7 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
     while (rest) {
       const int i = wd * 32 + __ffs(rest) - 1;
       rest &= rest - 1;
-      const uint32_t key = keys[key_slot(base + i)];
+      const uint32_t key = keys[key_slot4(base + i)];
       if (key > T) m_gt[wd] |= 1u << (i & 31);
       else if (key == T) m_eq[wd] |= 1u << (i & 31);
     }
@@ -660,8 +695,8 @@ __global__ void iota_kernel(int32_t* out, int rows, int n, int row_stride) {
 
 }  // namespace
 
-static inline int key_slot_host(int j) { return j + (j >> 5); }
-constexpr int FAST_SMEM_BYTES = (SEL_SMEM_KEYS + SEL_SMEM_KEYS / 32 + 64) * 4;
+static inline int key_slot4_host(int j) { return j + ((j >> 5) << 2); }
+constexpr int FAST_SMEM_BYTES = (FAST_MAX_KEYS + FAST_MAX_KEYS / 8 + 64) * 4;
 
 bool select_needs_scratch(int n) { return n > SEL_SMEM_KEYS; }
 
@@ -694,9 +729,9 @@ cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel
     attr_done = true;
   }
   const int r = pool_kernel >> 1;
-  if (n <= SEL_SMEM_KEYS && r <= 7) {
+  if (n <= FAST_MAX_KEYS && r <= 7) {
     const int ept = (((n + SEL_THREADS - 1) / SEL_THREADS) + 7) & ~7;
-    const int words = key_slot_host(SEL_THREADS * ept) + 1;
+    const int words = key_slot4_host(SEL_THREADS * ept) + 4;
 #define SNAPKV_FAST_LAUNCH(RM, P)                                                            \
   pool_topk_fast_kernel<RM, P><<<rows, SEL_THREADS, words * 4, stream>>>(vote, n, r, pool_type, \
                                                                         ept, ksel, out_idx)

@@ -94,6 +94,11 @@ def test_uniform_attention_closed_form_on_gpu():
     (2, 60001, 5, "avg", 1000),
     (1, 7, 7, "avg", 3),
     (2, 3000, 63, "max", 1500),
+    (2, 40960, 5, "avg", 4064),     # longest row of the vectorised one-CTA kernel (40 keys a thread)
+    (2, 40961, 7, "max", 4064),     # one more: generic one-CTA kernel, keys still on chip
+    (1, 49152, 13, "max", 8128),
+    (3, 32736, 13, "avg", 4064),    # radius 6 with its own instantiation
+    (2, 16352, 3, "max", 992),      # radius 1: run-time radius path
 ])
 def test_pool_topk_matches_oracle(rows, n, kernel, ptype, ksel):
     g = torch.Generator().manual_seed(n + kernel)
