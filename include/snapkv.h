@@ -150,8 +150,16 @@ snapkv_status_t snapkv_gather(const void* k, const void* v, const int32_t* idx,
  * with the shapes above (out_k/out_v [B,Hq,budget,d], out_idx [B,Hq,budget-W]).
  * `staging` is DEVICE scratch of at least snapkv_host_staging_size(...) bytes,
  * 256-byte aligned, holding the device copies and the workspace.  Copies in,
- * compresses, copies out, all on `stream`; returns after enqueueing (synchronise
- * the stream before reading the outputs).
+ * compresses, copies out; returns after enqueueing (synchronise `stream` before
+ * reading the outputs).  The (batch, KV head) pairs are independent (Sec. 4.1: every
+ * head selects on its own), so they go through in up to eight parts: a part's
+ * results are copied back on a side stream of the library while the next part's
+ * inputs are still arriving on `stream`, and `stream` waits for the last copy back
+ * before the call's work counts as complete.  The side stream and its events are
+ * created on the first call on a device and kept for the life of the process (make
+ * that first call outside any stream capture); if they cannot be created everything
+ * runs on `stream`.  The status block (snapkv_device_status on the workspace part of
+ * `staging`) keeps the first error of any part.
  */
 size_t snapkv_host_staging_size(int B, int Hq, int Hkv, int L, int d, int W,
                                 int pool_kernel, int pool_type, int budget);

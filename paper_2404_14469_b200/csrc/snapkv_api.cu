@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/snapkv.h"
 #include "launch.cuh"
 #include "snapkv_internal.h"
@@ -20,11 +22,15 @@ __global__ void clear_kernel(uint4* p, int n16) {
     p[i] = make_uint4(0u, 0u, 0u, 0u);
 }
 
-static cudaError_t launch_clear(uint8_t* ws, const WorkspaceLayout& w, cudaStream_t s) {
-  const int n16 = static_cast<int>((w.off_partials - w.off_status) / 16);
+// `keep_status`: leave the status block alone (a later part of one logical call must not wipe
+// an error an earlier part recorded) and clear the counters only.
+static cudaError_t launch_clear(uint8_t* ws, const WorkspaceLayout& w, cudaStream_t s,
+                                bool keep_status = false) {
+  const size_t from = keep_status ? w.off_counters : w.off_status;
+  const int n16 = static_cast<int>((w.off_partials - from) / 16);
   const int blocks = n16 > 256 * 64 ? 64 : (n16 + 255) / 256;
   return launch_pdl(clear_kernel, dim3(blocks), dim3(256), 0, s,
-                    reinterpret_cast<uint4*>(ws + w.off_status), n16);
+                    reinterpret_cast<uint4*>(ws + from), n16);
 }
 
 WorkspaceLayout make_layout(const ScorePlan& p, int B, int Hq, int n, bool need_vote,
@@ -49,6 +55,38 @@ WorkspaceLayout make_layout(const ScorePlan& p, int B, int Hq, int n, bool need_
 }
 
 static thread_local int g_last_launches = 0;
+
+// Side stream and events of snapkv_compress_host, one set per device, created on first use
+// and kept for the life of the process (nullptr if they cannot be created: the entry point
+// then copies back on the caller's stream).
+constexpr int HOST_PARTS = 8;
+struct HostSide {
+  cudaStream_t stream;
+  cudaEvent_t computed[HOST_PARTS];
+  cudaEvent_t done;
+};
+static HostSide* host_side() {
+  constexpr int MAX_DEV = 64;
+  static std::mutex mu;
+  static HostSide* table[MAX_DEV] = {};
+  static bool failed[MAX_DEV] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEV) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (table[dev] || failed[dev]) return table[dev];
+  HostSide* h = new HostSide();
+  bool ok = cudaStreamCreateWithFlags(&h->stream, cudaStreamNonBlocking) == cudaSuccess;
+  for (int i = 0; ok && i < HOST_PARTS; ++i)
+    ok = cudaEventCreateWithFlags(&h->computed[i], cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&h->done, cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) {
+    failed[dev] = true;
+    delete h;
+    return nullptr;
+  }
+  table[dev] = h;
+  return h;
+}
 
 static snapkv_status_t check_common(int B, int Hq, int Hkv, int L, int d, int W) {
   if (B < 1 || Hq < 1 || Hkv < 1 || L < 1 || d < 1 || W < 1) return SNAPKV_ERR_INVALID_ARG;
@@ -166,10 +204,11 @@ snapkv_status_t snapkv_gather(const void* k, const void* v, const int32_t* idx, 
   return e == cudaSuccess ? SNAPKV_OK : SNAPKV_ERR_CUDA;
 }
 
-snapkv_status_t snapkv_compress(const void* q_obs, const void* k, const void* v, int B, int Hq,
-                                int Hkv, int L, int d, int W, int pool_kernel, int pool_type,
-                                int budget, void* out_k, void* out_v, int32_t* out_idx,
-                                void* workspace, size_t workspace_bytes, void* stream) {
+static snapkv_status_t compress_impl(const void* q_obs, const void* k, const void* v, int B, int Hq,
+                                     int Hkv, int L, int d, int W, int pool_kernel, int pool_type,
+                                     int budget, void* out_k, void* out_v, int32_t* out_idx,
+                                     void* workspace, size_t workspace_bytes, void* stream,
+                                     bool keep_status) {
   snapkv_status_t st = check_common(B, Hq, Hkv, L, d, W);
   if (st != SNAPKV_OK) return st;
   st = check_pool(pool_kernel, pool_type);
@@ -199,7 +238,7 @@ snapkv_status_t snapkv_compress(const void* q_obs, const void* k, const void* v,
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < w.total)
     return SNAPKV_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  if (launch_clear(ws, w, s) != cudaSuccess) return SNAPKV_ERR_CUDA;
+  if (launch_clear(ws, w, s, keep_status) != cudaSuccess) return SNAPKV_ERR_CUDA;
   launches += 1;
   float* vote = reinterpret_cast<float*>(ws + w.off_vote);
   const int ksel = budget - W;
@@ -220,6 +259,14 @@ snapkv_status_t snapkv_compress(const void* q_obs, const void* k, const void* v,
   return SNAPKV_OK;
 }
 
+snapkv_status_t snapkv_compress(const void* q_obs, const void* k, const void* v, int B, int Hq,
+                                int Hkv, int L, int d, int W, int pool_kernel, int pool_type,
+                                int budget, void* out_k, void* out_v, int32_t* out_idx,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  return compress_impl(q_obs, k, v, B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget, out_k,
+                       out_v, out_idx, workspace, workspace_bytes, stream, false);
+}
+
 size_t snapkv_host_staging_size(int B, int Hq, int Hkv, int L, int d, int W, int pool_kernel,
                                 int pool_type, int budget) {
   if (check_common(B, Hq, Hkv, L, d, W) != SNAPKV_OK) return 0;
@@ -229,7 +276,20 @@ size_t snapkv_host_staging_size(int B, int Hq, int Hkv, int L, int d, int W, int
   const size_t ob = align_up(static_cast<size_t>(B) * Hq * budget * d * 2, 256);
   const size_t ib = align_up(static_cast<size_t>(B) * Hq * (budget - W) * 4, 256);
   size_t ws = 0;
-  if (budget < L) ws = snapkv_workspace_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget);
+  if (budget < L) {
+    // the entry point works through the (batch, KV head) pairs in parts, each a problem of
+    // its own; the workspace must hold the largest of them (and the whole, if it runs as one)
+    ws = snapkv_workspace_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget);
+    const int pairs = B * Hkv, g = Hq / Hkv;
+    const int parts = pairs < HOST_PARTS ? pairs : HOST_PARTS;
+    const int per = (pairs + parts - 1) / parts;
+    const int sizes[2] = {per, pairs % per};
+    for (int np : sizes)
+      if (np > 0) {
+        const size_t w1 = snapkv_workspace_size(1, np * g, np, L, d, W, pool_kernel, pool_type, budget);
+        if (w1 > ws) ws = w1;
+      }
+  }
   return qb + 2 * kb + 2 * ob + ib + align_up(ws, 256);
 }
 
@@ -262,18 +322,56 @@ snapkv_status_t snapkv_compress_host(const void* q_obs, const void* k, const voi
   uint8_t* dws = p;
   const size_t ws_bytes = staging_bytes - static_cast<size_t>(dws - static_cast<uint8_t*>(staging));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (cudaMemcpyAsync(dq, q_obs, q_raw, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(dk, k, k_raw, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(dv, v, k_raw, cudaMemcpyHostToDevice, s) != cudaSuccess)
-    return SNAPKV_ERR_CUDA;
-  snapkv_status_t st =
-      snapkv_compress(dq, dk, dv, B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget, dok, dov,
-                      reinterpret_cast<int32_t*>(di), dws, ws_bytes, stream);
-  if (st != SNAPKV_OK) return st;
-  if (cudaMemcpyAsync(out_k, dok, o_raw, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-      cudaMemcpyAsync(out_v, dov, o_raw, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-      cudaMemcpyAsync(out_idx, di, i_raw, cudaMemcpyDeviceToHost, s) != cudaSuccess)
-    return SNAPKV_ERR_CUDA;
+  // The (batch, KV head) pairs are independent: they go through in up to HOST_PARTS parts so
+  // that the copy back of one part (on a side stream) runs while the next part's inputs are
+  // still coming in; PCIe carries both directions at once.
+  const int pairs = B * Hkv, g = Hq / Hkv;
+  HostSide* side = host_side();
+  int parts = side ? (pairs < HOST_PARTS ? pairs : HOST_PARTS) : 1;
+  const int per = (pairs + parts - 1) / parts;
+  parts = (pairs + per - 1) / per;
+  const size_t q_pair = static_cast<size_t>(g) * W * d * 2, k_pair = static_cast<size_t>(L) * d * 2;
+  const size_t o_pair = static_cast<size_t>(g) * budget * d * 2;
+  const size_t i_pair = static_cast<size_t>(g) * (budget - W) * 4;
+  int launches = 0;
+  for (int c = 0; c < parts; ++c) {
+    const int p0 = c * per, np = (pairs - p0 < per) ? pairs - p0 : per;
+    const size_t qo = p0 * q_pair, ko = p0 * k_pair, oo = p0 * o_pair, io = p0 * i_pair;
+    if (cudaMemcpyAsync(dq + qo, static_cast<const uint8_t*>(q_obs) + qo, np * q_pair,
+                        cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(dk + ko, static_cast<const uint8_t*>(k) + ko, np * k_pair,
+                        cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(dv + ko, static_cast<const uint8_t*>(v) + ko, np * k_pair,
+                        cudaMemcpyHostToDevice, s) != cudaSuccess)
+      return SNAPKV_ERR_CUDA;
+    // one part is a problem of its own with batch 1 and np KV heads (the layouts are flat
+    // over batch and KV head); the parts share the workspace, which the stream serialises
+    const snapkv_status_t st = compress_impl(
+        dq + qo, dk + ko, dv + ko, 1, np * g, np, L, d, W, pool_kernel, pool_type, budget,
+        dok + oo, dov + oo, reinterpret_cast<int32_t*>(di + io), dws, ws_bytes, stream, c > 0);
+    if (st != SNAPKV_OK) return st;
+    launches += g_last_launches;
+    cudaStream_t back = s;
+    if (side) {
+      if (cudaEventRecord(side->computed[c], s) != cudaSuccess ||
+          cudaStreamWaitEvent(side->stream, side->computed[c], 0) != cudaSuccess)
+        return SNAPKV_ERR_CUDA;
+      back = side->stream;
+    }
+    if (cudaMemcpyAsync(static_cast<uint8_t*>(out_k) + oo, dok + oo, np * o_pair,
+                        cudaMemcpyDeviceToHost, back) != cudaSuccess ||
+        cudaMemcpyAsync(static_cast<uint8_t*>(out_v) + oo, dov + oo, np * o_pair,
+                        cudaMemcpyDeviceToHost, back) != cudaSuccess ||
+        cudaMemcpyAsync(reinterpret_cast<uint8_t*>(out_idx) + io, di + io, np * i_pair,
+                        cudaMemcpyDeviceToHost, back) != cudaSuccess)
+      return SNAPKV_ERR_CUDA;
+  }
+  if (side) {  // the caller's stream is complete only when the last copy back is
+    if (cudaEventRecord(side->done, side->stream) != cudaSuccess ||
+        cudaStreamWaitEvent(s, side->done, 0) != cudaSuccess)
+      return SNAPKV_ERR_CUDA;
+  }
+  g_last_launches = launches;
   return SNAPKV_OK;
 }
 

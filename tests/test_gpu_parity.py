@@ -273,6 +273,30 @@ def test_compress_from_host_buffers():
     assert torch.equal(ok, ref[0].cpu()) and torch.equal(ov, ref[1].cpu()) and torch.equal(oi, ref[2].cpu())
 
 
+@pytest.mark.parametrize("B,Hq,Hkv,L,d,W,kernel,budget", [
+    (3, 8, 2, 700, 128, 16, 5, 128),     # 6 (batch, KV head) pairs, one per part
+    (1, 22, 11, 900, 64, 32, 7, 300),    # 11 pairs: five parts of two and one of one
+    (2, 4, 4, 300, 128, 32, 7, 300),     # budget >= L: identity, expanded to Hq heads
+    (1, 2, 1, 4000, 128, 64, 13, 1000),  # one pair: a single part
+])
+def test_compress_from_host_buffers_in_parts(B, Hq, Hkv, L, d, W, kernel, budget):
+    data = synth.make_random(B, Hq, Hkv, L, d, W, seed=21)
+    rows = min(budget, L)
+    q, k, v = (data[x].pin_memory() for x in ("q_obs", "k", "v"))
+    dev = _to_dev(data)
+    ref = sk.snapkv_compress(dev["q_obs"], dev["k"], dev["v"], kernel, sk.POOL_MAX, budget)
+    need = sk.snapkv_host_staging_size(B, Hq, Hkv, L, d, W, kernel, 0, rows)
+    staging = torch.empty(need, dtype=torch.uint8, device="cuda")
+    for _ in range(2):  # the second call reuses the library's side stream and events
+        ok = torch.zeros(B, Hq, rows, d, dtype=torch.bfloat16).pin_memory()
+        ov = torch.zeros_like(ok).pin_memory()
+        oi = torch.zeros(B, Hq, rows - W, dtype=torch.int32).pin_memory()
+        sk.snapkv_compress_host(q, k, v, kernel, sk.POOL_MAX, budget, ok, ov, oi, staging)
+        torch.cuda.current_stream().synchronize()  # the caller's stream alone covers the copies back
+        assert torch.equal(ok, ref[0].cpu()) and torch.equal(ov, ref[1].cpu())
+        assert torch.equal(oi, ref[2].cpu())
+
+
 # ------------------------------------------------------------------ full-size workloads, sampled heads
 def _sample_heads(B, Hq, count, seed):
     g = torch.Generator().manual_seed(seed)
