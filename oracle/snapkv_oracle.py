@@ -94,6 +94,43 @@ def window_votes(q_head: np.ndarray, k_head: np.ndarray) -> np.ndarray:
     return vote_from_probs(window_softmax(window_logits(q_head, k_head)))
 
 
+def window_lse(s: np.ndarray) -> np.ndarray:
+    """Natural-log sum-exp of every window row over the keys it sees (the normaliser of
+    Sec. 4's softmax, as a prefill attention kernel would hand it on): [W, L] -> [W]."""
+    W, L = s.shape
+    n = L - W
+    out = np.empty(W, dtype=np.float64)
+    for i in range(W):
+        row = s[i, : n + i + 1]
+        m = row.max()
+        out[i] = m + math.log(np.exp(row - m).sum())
+    return out
+
+
+def votes_given_lse(s: np.ndarray, lse: np.ndarray) -> np.ndarray:
+    """Eq. 1 with the normaliser supplied: C[j] = sum_i exp(s[i, j] - lse[i]) over the W
+    window rows, prefix columns only (every prefix key is visible to every window row).
+    Not in the paper's listing, which recomputes the softmax; same result when `lse` is
+    the rows' own log-sum-exp."""
+    W, L = s.shape
+    n = L - W
+    return np.exp(s[:, :n] - lse[:, None]).sum(axis=0)
+
+
+def lse_obs(q_obs: np.ndarray, k: np.ndarray) -> np.ndarray:
+    """window_lse for every (batch, query head): bf16 bits in, fp64 [B, Hq, W] out."""
+    B, Hq, W, d = q_obs.shape
+    _, Hkv, L, _ = k.shape
+    g = Hq // Hkv
+    out = np.empty((B, Hq, W), dtype=np.float64)
+    for b in range(B):
+        for c in range(Hkv):
+            kf = bf16_bits_to_f64(k[b, c])
+            for h in range(c * g, (c + 1) * g):
+                out[b, h] = window_lse(window_logits(bf16_bits_to_f64(q_obs[b, h]), kf))
+    return out
+
+
 def pool1d(vote: np.ndarray, pool_kernel: int, pool_type: int) -> np.ndarray:
     """Listing 1's pool1d(kernel_size, padding=kernel_size//2, stride=1) on one row.
 
@@ -169,7 +206,7 @@ def votes(q_obs: np.ndarray, k: np.ndarray, workers: int = 1) -> np.ndarray:
 
 
 def compress(q_obs: np.ndarray, k: np.ndarray, v: np.ndarray, pool_kernel: int,
-             pool_type: int, budget: int, workers: int = 1, heads=None):
+             pool_type: int, budget: int, workers: int = 1, heads=None, lse=None):
     """The whole step (Listing 1) on bf16 bit patterns.
 
     Returns a dict with
@@ -178,6 +215,8 @@ def compress(q_obs: np.ndarray, k: np.ndarray, v: np.ndarray, pool_kernel: int,
       vote, pooled : fp64   [B, Hq, n] (None on the identity path)
     `heads` optionally restricts the work to a list of (b, h) pairs (other heads
     are left zero) so that sampled checks at large sizes stay affordable.
+    `lse` (fp64 [B, Hq, W]) switches to the supplied-normaliser variant: votes are
+    votes_given_lse instead of window_votes; everything after the vote is the same.
     """
     B, Hq, Hkv, L, d, W = _check_shapes(q_obs, k, v)
     if budget <= W:
@@ -209,7 +248,10 @@ def compress(q_obs: np.ndarray, k: np.ndarray, v: np.ndarray, pool_kernel: int,
             return
         kf = bf16_bits_to_f64(k[b, c])
         for h in hs:
-            vt = window_votes(bf16_bits_to_f64(q_obs[b, h]), kf)
+            if lse is None:
+                vt = window_votes(bf16_bits_to_f64(q_obs[b, h]), kf)
+            else:
+                vt = votes_given_lse(window_logits(bf16_bits_to_f64(q_obs[b, h]), kf), lse[b, h])
             pv = pool1d(vt, pool_kernel, pool_type)
             idx = topk_positions(pv, ksel)
             vote[b, h] = vt
