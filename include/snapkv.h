@@ -145,6 +145,33 @@ snapkv_status_t snapkv_gather(const void* k, const void* v, const int32_t* idx,
                               void* out_k, void* out_v, void* stream);
 
 /*
+ * Supplied-normaliser variant of snapkv_window_scores and snapkv_compress.  The paper's
+ * listing recomputes the window rows' softmax after the prompt phase (Listing 1,
+ * compute_attn), although the attention kernel of the prompt phase already held each
+ * row's normaliser.  Here the caller passes it in: lse_obs, DEVICE fp32 [B, Hq, W],
+ * lse_obs[b,h,i] = natural log of the sum over the keys j <= L - W + i of
+ * exp(q_obs[b,h,i] . k[b,kv(h),j] / sqrt(d)) (the log-sum-exp flash-attention style
+ * kernels return).  Votes are then vote[j] = sum_i exp(logit[i,j] - lse_obs[i]) (Eq. 1
+ * with the softmax written out), computed in ONE sweep over K: no statistics pass, half
+ * of the exponentials and of the K traffic.  Everything after the vote (pooling, top-k,
+ * gather) is the same as in snapkv_compress; with the rows' true log-sum-exp the results
+ * agree with it to rounding.  Same arguments, workspace size, errors and ownership as the
+ * functions they mirror; lse_obs is read only, must be 4-byte aligned and is consumed by
+ * the time the stream's work completes.  A wrong lse_obs scales that row's contribution;
+ * nothing checks it.
+ */
+snapkv_status_t snapkv_window_scores_lse(const void* q_obs, const void* k, const float* lse_obs,
+                                         int B, int Hq, int Hkv, int L, int d, int W,
+                                         float* out_vote, void* workspace,
+                                         size_t workspace_bytes, void* stream);
+snapkv_status_t snapkv_compress_lse(const void* q_obs, const void* k, const void* v,
+                                    const float* lse_obs,
+                                    int B, int Hq, int Hkv, int L, int d, int W,
+                                    int pool_kernel, int pool_type, int budget,
+                                    void* out_k, void* out_v, int32_t* out_idx,
+                                    void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * snapkv_compress for callers whose tensors live in host memory (pinned memory
  * gives asynchronous copies).  q_obs, k, v, out_k, out_v, out_idx are HOST pointers
  * with the shapes above (out_k/out_v [B,Hq,budget,d], out_idx [B,Hq,budget-W]).

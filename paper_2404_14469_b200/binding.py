@@ -25,6 +25,7 @@ SYMBOLS = [
     "snapkv_window_scores", "snapkv_pool_topk_workspace_size", "snapkv_pool_topk", "snapkv_gather",
     "snapkv_host_staging_size", "snapkv_compress_host", "snapkv_device_status",
     "snapkv_last_launch_count", "snapkv_pool_topk_static",
+    "snapkv_window_scores_lse", "snapkv_compress_lse",
 ]
 
 _lib = None
@@ -55,6 +56,10 @@ def lib() -> ctypes.CDLL:
     L.snapkv_compress.argtypes = [c_vp] * 3 + [c_int] * 9 + [c_vp] * 3 + [c_vp, c_sz, c_vp]
     L.snapkv_window_scores.restype = c_int
     L.snapkv_window_scores.argtypes = [c_vp] * 2 + [c_int] * 6 + [c_vp, c_vp, c_sz, c_vp]
+    L.snapkv_window_scores_lse.restype = c_int
+    L.snapkv_window_scores_lse.argtypes = [c_vp] * 3 + [c_int] * 6 + [c_vp, c_vp, c_sz, c_vp]
+    L.snapkv_compress_lse.restype = c_int
+    L.snapkv_compress_lse.argtypes = [c_vp] * 4 + [c_int] * 9 + [c_vp] * 3 + [c_vp, c_sz, c_vp]
     L.snapkv_pool_topk_workspace_size.restype = c_sz
     L.snapkv_pool_topk_workspace_size.argtypes = [c_int, c_int]
     L.snapkv_pool_topk.restype = c_int
@@ -114,8 +119,22 @@ def snapkv_workspace_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget) -
     return lib().snapkv_workspace_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget)
 
 
+def _lse_arg(lse_obs, B, Hq, W):
+    if not (lse_obs.is_cuda and lse_obs.dtype == torch.float32 and lse_obs.is_contiguous()
+            and tuple(lse_obs.shape) == (B, Hq, W)):
+        raise SnapKVError("lse_obs must be a contiguous CUDA fp32 [B, Hq, W] tensor")
+    return lse_obs.data_ptr()
+
+
+def snapkv_compress_lse(q_obs, k, v, lse_obs, pool_kernel: int, pool_type: int, budget: int,
+                        out_k=None, out_v=None, out_idx=None, workspace=None):
+    """snapkv_compress with the window rows' log-sum-exp supplied (fp32 [B, Hq, W])."""
+    return snapkv_compress(q_obs, k, v, pool_kernel, pool_type, budget, out_k, out_v, out_idx,
+                           workspace, lse_obs=lse_obs)
+
+
 def snapkv_compress(q_obs, k, v, pool_kernel: int, pool_type: int, budget: int,
-                    out_k=None, out_v=None, out_idx=None, workspace=None):
+                    out_k=None, out_v=None, out_idx=None, workspace=None, lse_obs=None):
     """Whole step on device tensors.  Returns (out_k, out_v, out_idx, workspace).
 
     out_k/out_v: bf16 [B, Hq, min(budget, L), d]; out_idx: int32 [B, Hq, rows - W].
@@ -137,15 +156,24 @@ def snapkv_compress(q_obs, k, v, pool_kernel: int, pool_type: int, budget: int,
     need = L_.snapkv_workspace_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, eff_budget)
     if workspace is None or workspace.numel() < need:
         workspace = _alloc_ws(need, dev)
-    code = L_.snapkv_compress(q_obs.data_ptr(), k.data_ptr(), v.data_ptr(), B, Hq, Hkv, L, d, W,
-                              pool_kernel, pool_type, eff_budget, out_k.data_ptr(), out_v.data_ptr(),
-                              out_idx.data_ptr(), workspace.data_ptr(), workspace.numel(),
-                              _stream_ptr())
+    tail = (B, Hq, Hkv, L, d, W, pool_kernel, pool_type, eff_budget, out_k.data_ptr(),
+            out_v.data_ptr(), out_idx.data_ptr(), workspace.data_ptr(), workspace.numel(),
+            _stream_ptr())
+    if lse_obs is None:
+        code = L_.snapkv_compress(q_obs.data_ptr(), k.data_ptr(), v.data_ptr(), *tail)
+    else:
+        code = L_.snapkv_compress_lse(q_obs.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                      _lse_arg(lse_obs, B, Hq, W), *tail)
     _check(code, "snapkv_compress")
     return out_k, out_v, out_idx, workspace
 
 
-def snapkv_window_scores(q_obs, k, out_vote=None, workspace=None):
+def snapkv_window_scores_lse(q_obs, k, lse_obs, out_vote=None, workspace=None):
+    """snapkv_window_scores with the window rows' log-sum-exp supplied (fp32 [B, Hq, W])."""
+    return snapkv_window_scores(q_obs, k, out_vote, workspace, lse_obs=lse_obs)
+
+
+def snapkv_window_scores(q_obs, k, out_vote=None, workspace=None, lse_obs=None):
     """Votes fp32 [B, Hq, n].  Returns (out_vote, workspace)."""
     _dev_bf16(q_obs, "q_obs"), _dev_bf16(k, "k")
     B, Hq, Hkv, L, d, W = _shapes(q_obs, k)
@@ -156,9 +184,13 @@ def snapkv_window_scores(q_obs, k, out_vote=None, workspace=None):
     need = L_.snapkv_workspace_size(B, Hq, Hkv, L, d, W, 1, 0, W + 1)
     if workspace is None or workspace.numel() < need:
         workspace = _alloc_ws(need, dev)
-    code = L_.snapkv_window_scores(q_obs.data_ptr(), k.data_ptr(), B, Hq, Hkv, L, d, W,
-                                   out_vote.data_ptr(), workspace.data_ptr(), workspace.numel(),
-                                   _stream_ptr())
+    tail = (B, Hq, Hkv, L, d, W, out_vote.data_ptr(), workspace.data_ptr(), workspace.numel(),
+            _stream_ptr())
+    if lse_obs is None:
+        code = L_.snapkv_window_scores(q_obs.data_ptr(), k.data_ptr(), *tail)
+    else:
+        code = L_.snapkv_window_scores_lse(q_obs.data_ptr(), k.data_ptr(),
+                                           _lse_arg(lse_obs, B, Hq, W), *tail)
     _check(code, "snapkv_window_scores")
     return out_vote, workspace
 

@@ -145,9 +145,10 @@ size_t snapkv_pool_topk_workspace_size(int rows, int n) {
   return select_scratch_bytes(rows, n);
 }
 
-snapkv_status_t snapkv_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv,
-                                     int L, int d, int W, float* out_vote, void* workspace,
-                                     size_t workspace_bytes, void* stream) {
+static snapkv_status_t window_scores_impl(const void* q_obs, const void* k, const float* lse_obs,
+                                          int B, int Hq, int Hkv, int L, int d, int W,
+                                          float* out_vote, void* workspace,
+                                          size_t workspace_bytes, void* stream) {
   snapkv_status_t st = check_common(B, Hq, Hkv, L, d, W);
   if (st != SNAPKV_OK) return st;
   if (W >= L) return SNAPKV_ERR_INVALID_ARG;
@@ -166,10 +167,26 @@ snapkv_status_t snapkv_window_scores(const void* q_obs, const void* k, int B, in
   cudaError_t e = launch_window_scores(
       q_obs, k, B, Hq, Hkv, L, d, W, p, out_vote, reinterpret_cast<int*>(ws + w.off_status),
       reinterpret_cast<int*>(ws + w.off_counters), reinterpret_cast<float*>(ws + w.off_partials),
-      reinterpret_cast<float*>(ws + w.off_lse), s, &launches);
+      reinterpret_cast<float*>(ws + w.off_lse), s, &launches, lse_obs);
   if (e != cudaSuccess) return SNAPKV_ERR_CUDA;
   g_last_launches = launches;
   return SNAPKV_OK;
+}
+
+snapkv_status_t snapkv_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv,
+                                     int L, int d, int W, float* out_vote, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+  return window_scores_impl(q_obs, k, nullptr, B, Hq, Hkv, L, d, W, out_vote, workspace,
+                            workspace_bytes, stream);
+}
+
+snapkv_status_t snapkv_window_scores_lse(const void* q_obs, const void* k, const float* lse_obs,
+                                         int B, int Hq, int Hkv, int L, int d, int W,
+                                         float* out_vote, void* workspace, size_t workspace_bytes,
+                                         void* stream) {
+  if (!lse_obs || (reinterpret_cast<uintptr_t>(lse_obs) & 3)) return SNAPKV_ERR_INVALID_ARG;
+  return window_scores_impl(q_obs, k, lse_obs, B, Hq, Hkv, L, d, W, out_vote, workspace,
+                            workspace_bytes, stream);
 }
 
 snapkv_status_t snapkv_pool_topk(const float* vote, int rows, int n, int pool_kernel, int pool_type,
@@ -208,7 +225,7 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
                                      int Hkv, int L, int d, int W, int pool_kernel, int pool_type,
                                      int budget, void* out_k, void* out_v, int32_t* out_idx,
                                      void* workspace, size_t workspace_bytes, void* stream,
-                                     bool keep_status) {
+                                     bool keep_status, const float* lse_obs = nullptr) {
   snapkv_status_t st = check_common(B, Hq, Hkv, L, d, W);
   if (st != SNAPKV_OK) return st;
   st = check_pool(pool_kernel, pool_type);
@@ -246,7 +263,8 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
                            reinterpret_cast<int*>(ws + w.off_status),
                            reinterpret_cast<int*>(ws + w.off_counters),
                            reinterpret_cast<float*>(ws + w.off_partials),
-                           reinterpret_cast<float*>(ws + w.off_lse), s, &launches) != cudaSuccess)
+                           reinterpret_cast<float*>(ws + w.off_lse), s, &launches, lse_obs) !=
+      cudaSuccess)
     return SNAPKV_ERR_CUDA;
   if (launch_pool_topk(vote, B * Hq, n, pool_kernel, pool_type, ksel, out_idx,
                        scratch ? reinterpret_cast<float*>(ws + w.off_pooled) : nullptr, s,
@@ -265,6 +283,16 @@ snapkv_status_t snapkv_compress(const void* q_obs, const void* k, const void* v,
                                 void* workspace, size_t workspace_bytes, void* stream) {
   return compress_impl(q_obs, k, v, B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget, out_k,
                        out_v, out_idx, workspace, workspace_bytes, stream, false);
+}
+
+snapkv_status_t snapkv_compress_lse(const void* q_obs, const void* k, const void* v,
+                                    const float* lse_obs, int B, int Hq, int Hkv, int L, int d,
+                                    int W, int pool_kernel, int pool_type, int budget, void* out_k,
+                                    void* out_v, int32_t* out_idx, void* workspace,
+                                    size_t workspace_bytes, void* stream) {
+  if (!lse_obs || (reinterpret_cast<uintptr_t>(lse_obs) & 3)) return SNAPKV_ERR_INVALID_ARG;
+  return compress_impl(q_obs, k, v, B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget, out_k,
+                       out_v, out_idx, workspace, workspace_bytes, stream, false, lse_obs);
 }
 
 size_t snapkv_host_staging_size(int B, int Hq, int Hkv, int L, int d, int W, int pool_kernel,

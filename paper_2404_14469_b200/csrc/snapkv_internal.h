@@ -57,11 +57,13 @@ bool select_needs_scratch(int n);
 size_t select_scratch_bytes(int rows, int n);  // 0 when the rows fit one CTA
 
 // Enqueue both scoring passes.  `vote` is fp32 [B*Hq, n].  `counters` must be zero when the
-// kernel starts (the callers clear it together with the status block).
+// kernel starts (the callers clear it together with the status block).  With `lse_obs`
+// (device fp32 [B*Hq, W], natural-log sum-exp of every window row) the statistics pass is
+// skipped: a small kernel converts the rows first, then only the vote pass runs.
 cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv, int L,
                                  int d, int W, const ScorePlan& plan, float* vote, int* status,
                                  int* counters, float* partials, float* lse2, cudaStream_t stream,
-                                 int* launches);
+                                 int* launches, const float* lse_obs = nullptr);
 
 // Pool + top-k over `rows` rows of fp32 votes.  `pooled_scratch` (select_scratch_bytes bytes)
 // is only touched when select_needs_scratch(n).

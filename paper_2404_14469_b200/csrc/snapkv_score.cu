@@ -74,6 +74,7 @@ struct ScoreArgs {
   int T1, T2;               // tiles per unit in the statistics / vote pass
   int maxseg;               // partial slots per unit
   int pipelined;            // how many waves the statistics run ahead of the votes (>= 1)
+  int votes_only;           // 1: lse2 and the counters are already set, no statistics pass
   float c2;                 // log2(e) / sqrt(d)
   float* partials;          // [units][maxseg][MAX_COLS] log2-sum-exp of one CTA's share
   float* lse2;              // [units][MAX_COLS] minus the merged log2-sum-exp per window row
@@ -156,7 +157,7 @@ __device__ __forceinline__ void for_each_item(const ScoreArgs& a, int cta, int G
                                               F&& f) {
   // Phase order: statistics run `lag` waves ahead of votes: S(0) .. S(lag-1) V(0) S(lag)
   // V(1) ...; lag = 1 is the plain order S(0) V(0) S(1) V(1) ...
-  int s_next = 0, v_next = 0;
+  int s_next = a.votes_only ? a.nwaves : 0, v_next = 0;
   while (v_next < a.nwaves) {
     int w, vote;
     if (s_next < a.nwaves && s_next - v_next < lag) { w = s_next++; vote = 0; }
@@ -760,6 +761,29 @@ int sm_count() {
   return cached[dev];
 }
 
+// Supplied-normaliser variant: the caller hands in each window row's natural-log sum-exp
+// (what a prefill attention kernel keeps per query row).  This kernel puts it where the vote
+// pass expects the merged statistics - minus the log2-sum-exp, one row of MAX_COLS per unit -
+// and marks every unit as merged, so the scoring kernel runs its vote phases only.
+constexpr int COUNTER_READY = 1 << 30;
+__global__ void lse_prep_kernel(const float* __restrict__ lse_obs, float* __restrict__ lse2,
+                                int* __restrict__ counters, int units, int sub_per_kv, int g,
+                                int hpu, int W, int ncols) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int u = blockIdx.x, c = threadIdx.x;  // one block per unit, one thread per column
+  if (u >= units || c >= MAX_COLS) return;
+  const int ukv = u / sub_per_kv;
+  const int hq0 = ukv * g + (u - ukv * sub_per_kv) * hpu;  // flat over the batch
+  float out = 0.f;
+  if (c < ncols) {
+    const int hl = c / W, i = c - hl * W;
+    out = -lse_obs[static_cast<size_t>(hq0 + hl) * W + i] * 1.4426950408889634f;
+  }
+  lse2[static_cast<size_t>(u) * MAX_COLS + c] = out;
+  if (c == 0) counters[u] = COUNTER_READY;
+}
+
 template <int D, int NCH, bool SPLIT>
 cudaError_t run_scores(const CUtensorMap& tmK, const CUtensorMap& tmQ, const ScoreArgs& a,
                        int grid, cudaStream_t stream, int* launches) {
@@ -839,7 +863,7 @@ bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* pla
 cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv, int L,
                                  int d, int W, const ScorePlan& plan, float* vote, int* status,
                                  int* counters, float* partials, float* lse2, cudaStream_t stream,
-                                 int* launches) {
+                                 int* launches, const float* lse_obs) {
   CUtensorMap tmK, tmQ;
   {
     cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(L),
@@ -870,12 +894,20 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq
   a.T2 = plan.tiles_vote;
   a.maxseg = plan.maxseg;
   a.pipelined = plan.pipelined;
+  a.votes_only = lse_obs ? 1 : 0;
   a.c2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
   a.partials = partials;
   a.lse2 = lse2;
   a.counters = counters;
   a.status = status;
   a.vote = vote;
+  if (lse_obs) {
+    const cudaError_t e =
+        launch_pdl(lse_prep_kernel, dim3(plan.units), dim3(MAX_COLS), 0, stream, lse_obs, lse2,
+                   counters, plan.units, plan.sub_per_kv, plan.g, plan.hpu, W, plan.ncols);
+    if (e != cudaSuccess) return e;
+    *launches += 1;
+  }
   int grid = sm_count();
   if (grid > MAX_GRID) grid = MAX_GRID;
   const int nch = plan.npad >> 5;

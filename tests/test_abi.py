@@ -109,6 +109,20 @@ def test_other_entry_points_reject_bad_arguments(L):
     assert L.snapkv_compress_host(FAKE, FAKE, FAKE, 1, 4, 4, 1024, 96, 32, 7, 0, 256, FAKE, FAKE, FAKE,
                                   None, 0, None) == 2
     assert L.snapkv_device_status(None, None, None) == 1
+    # supplied-normaliser variant: a missing or misaligned lse_obs is an argument error,
+    # everything else is checked as in the functions it mirrors
+    assert L.snapkv_window_scores_lse(FAKE, FAKE, None, 1, 4, 4, 1024, 64, 32, FAKE, FAKE, 1 << 30,
+                                      None) == 1
+    assert L.snapkv_window_scores_lse(FAKE, FAKE, FAKE + 2, 1, 4, 4, 1024, 64, 32, FAKE, FAKE,
+                                      1 << 30, None) == 1
+    assert L.snapkv_window_scores_lse(FAKE, FAKE, FAKE, 1, 4, 4, 1024, 64, 32, FAKE, None, 0,
+                                      None) == 3
+    assert L.snapkv_compress_lse(FAKE, FAKE, FAKE, None, 1, 4, 4, 1024, 64, 32, 7, 0, 256, FAKE, FAKE,
+                                 FAKE, FAKE, 1 << 30, None) == 1
+    assert L.snapkv_compress_lse(FAKE, FAKE, FAKE, FAKE, 1, 4, 4, 1024, 64, 32, 6, 0, 256, FAKE, FAKE,
+                                 FAKE, FAKE, 1 << 30, None) == 1      # even pooling kernel
+    assert L.snapkv_compress_lse(FAKE, FAKE, FAKE, FAKE, 1, 4, 4, 1024, 64, 32, 7, 0, 256, FAKE, FAKE,
+                                 FAKE, None, 0, None) == 3
 
 
 def test_missing_library_fails_loudly(monkeypatch):
