@@ -186,6 +186,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--lse-in", action="store_true",
+                    help="time the supplied-normaliser variant (snapkv_compress_lse): the window "
+                         "rows' log-sum-exp is an input, K is swept once; not the paper's path")
     args = ap.parse_args()
 
     from paper_2404_14469_b200 import synth
@@ -231,11 +234,26 @@ def main():
     ws = torch.empty(sk.snapkv_workspace_size(w.B, w.Hq, w.Hkv, w.L, w.d, w.W, w.pool_kernel, ptype, budget),
                      dtype=torch.uint8, device=dev)
     vote = torch.empty(w.B * w.Hq, w.n, dtype=torch.float32, device=dev)
+    lses = [None] * layers
+    if args.lse_in:
+        # Input preparation for the variant, untimed: what the prompt phase's attention kernel
+        # would hand over.  Plain framework ops on the synthetic q and k; the library's own
+        # results with these inputs are checked against the oracle in tests/test_gpu_lse.py.
+        g = w.Hq // w.Hkv
+        pos = torch.arange(w.L, device=dev)[None, :] <= (w.n + torch.arange(w.W, device=dev))[:, None]
+        for i, (q, k, _) in enumerate(ins):
+            rows = []
+            for b in range(w.B):
+                kk = k[b].float().repeat_interleave(g, dim=0)                      # [Hq, L, d]
+                lg = torch.matmul(q[b].float(), kk.transpose(1, 2)) / (w.d ** 0.5)   # [Hq, W, L]
+                rows.append(torch.logsumexp(lg.masked_fill(~pos, float("-inf")), dim=-1))
+            lses[i] = torch.stack(rows).contiguous()
 
     def step():
         for i in range(layers):
             q, k, v = ins[i]
-            sk.snapkv_compress(q, k, v, w.pool_kernel, ptype, budget, out_k[i], out_v[i], out_idx[i], ws)
+            sk.snapkv_compress(q, k, v, w.pool_kernel, ptype, budget, out_k[i], out_v[i], out_idx[i], ws,
+                               lse_obs=lses[i])
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -275,7 +293,7 @@ def main():
             ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
             evs.append(ev)
             ev[0].record()
-            sk.snapkv_window_scores(q, k, vote.view(w.B, w.Hq, w.n), ws)
+            sk.snapkv_window_scores(q, k, vote.view(w.B, w.Hq, w.n), ws, lse_obs=lses[i])
             ev[1].record()
             sk.snapkv_pool_topk(vote, w.pool_kernel, ptype, ksel, out_idx[i].view(w.B * w.Hq, ksel), ws)
             ev[2].record()
@@ -295,11 +313,11 @@ def main():
     # scoring kernel is made resident while the clear kernel before it still runs, which an
     # event in between prevents).  Each layer has its own K: nothing is served from L2.
     e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sk.snapkv_window_scores(ins[0][0], ins[0][1], vote.view(w.B, w.Hq, w.n), ws)
+    sk.snapkv_window_scores(ins[0][0], ins[0][1], vote.view(w.B, w.Hq, w.n), ws, lse_obs=lses[0])
     e2.record()
     for _ in range(reps):
         for i in range(layers):
-            sk.snapkv_window_scores(ins[i][0], ins[i][1], vote.view(w.B, w.Hq, w.n), ws)
+            sk.snapkv_window_scores(ins[i][0], ins[i][1], vote.view(w.B, w.Hq, w.n), ws, lse_obs=lses[i])
     e3.record()
     torch.cuda.synchronize()
     stage_ms["score_with_events"] = stage_ms["score"]
@@ -319,10 +337,12 @@ def main():
     dom_bytes = ab[dom]
     achieved = dom_bytes / (stage_ms[dom] * 1e-3) / 1e9
     roofline = {
-        "bound": "hbm", "kernel": {"score": "score_kernel (statistics + vote passes)",
+        "bound": "hbm", "kernel": {"score": "score_kernel (vote pass only)" if args.lse_in
+                                    else "score_kernel (statistics + vote passes)",
                                     "gather": "gather_kernel"}[dom],
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC.get((dom, w.wid)),
+        "peak_kind": f"of {peak_kind}",
+        "traffic": None if args.lse_in else NCU_TRAFFIC.get((dom, w.wid)),
         "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": stage_ms[dom],
         "stage_ms_per_layer": stage_ms,
         "whole_step": {"algorithmic_bytes_per_layer": ab["total"], "ms_per_layer": ms_layer,
@@ -333,7 +353,7 @@ def main():
 
     # end to end through the host-buffer entry point: pinned host tensors in, pinned out
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not args.lse_in:
         q, k, v = (t.cpu().pin_memory() for t in ins[0])
         hk = torch.empty(w.B, w.Hq, budget, w.d, dtype=torch.bfloat16).pin_memory()
         hv = torch.empty_like(hk).pin_memory()
@@ -373,6 +393,9 @@ def main():
         cfg = workload_config(w, budget, layers)
         cfg["ms_per_layer"] = ms_layer
         cfg["parallelism"] = "replicas: each GPU compresses its own batch, no collective"
+        if args.lse_in:
+            cfg["variant"] = ("lse-in: the window rows' log-sum-exp is an input, one sweep over K "
+                              "(snapkv_compress_lse; not the paper's path)")
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,

@@ -28,6 +28,10 @@ Readings of points the paper leaves open (all listed again in the design notes):
   * ties in the top-k go to the lower position; indices are emitted ascending;
   * budget >= L is the identity.
 
+A variant outside the paper's listing is stated too: votes_given_lse / window_lse /
+lse_obs / compress(lse=...) take the window rows' log-sum-exp as an input (the prompt
+phase's attention kernel holds it) instead of recomputing the softmax.
+
 Every function here is pinned by tests that do not go through this file's own
 formulas (closed forms, invariants, library routines, brute force): see
 tests/test_oracle_*.py.  Nothing is "parity unpinned".
