@@ -162,8 +162,12 @@ static snapkv_status_t window_scores_impl(const void* q_obs, const void* k, cons
     return SNAPKV_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (launch_clear(ws, w, s) != cudaSuccess) return SNAPKV_ERR_CUDA;
-  int launches = 1;
+  // with a supplied normaliser the conversion kernel clears what the clear kernel would
+  int launches = 0;
+  if (!lse_obs) {
+    if (launch_clear(ws, w, s) != cudaSuccess) return SNAPKV_ERR_CUDA;
+    launches = 1;
+  }
   cudaError_t e = launch_window_scores(
       q_obs, k, B, Hq, Hkv, L, d, W, p, out_vote, reinterpret_cast<int*>(ws + w.off_status),
       reinterpret_cast<int*>(ws + w.off_counters), reinterpret_cast<float*>(ws + w.off_partials),
@@ -255,8 +259,10 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < w.total)
     return SNAPKV_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  if (launch_clear(ws, w, s, keep_status) != cudaSuccess) return SNAPKV_ERR_CUDA;
-  launches += 1;
+  if (!lse_obs) {
+    if (launch_clear(ws, w, s, keep_status) != cudaSuccess) return SNAPKV_ERR_CUDA;
+    launches += 1;
+  }
   float* vote = reinterpret_cast<float*>(ws + w.off_vote);
   const int ksel = budget - W;
   if (launch_window_scores(q_obs, k, B, Hq, Hkv, L, d, W, p, vote,

@@ -767,11 +767,13 @@ int sm_count() {
 // and marks every unit as merged, so the scoring kernel runs its vote phases only.
 constexpr int COUNTER_READY = 1 << 30;
 __global__ void lse_prep_kernel(const float* __restrict__ lse_obs, float* __restrict__ lse2,
-                                int* __restrict__ counters, int units, int sub_per_kv, int g,
-                                int hpu, int W, int ncols) {
+                                int* __restrict__ counters, int* __restrict__ status, int units,
+                                int sub_per_kv, int g, int hpu, int W, int ncols) {
   pdl_launch_dependents();
   pdl_wait();
   const int u = blockIdx.x, c = threadIdx.x;  // one block per unit, one thread per column
+  // this kernel stands in for the clear kernel of the two-sweep path: the status block too
+  if (u == 0 && c < STATUS_BYTES / 4) status[c] = 0;
   if (u >= units || c >= MAX_COLS) return;
   const int ukv = u / sub_per_kv;
   const int hq0 = ukv * g + (u - ukv * sub_per_kv) * hpu;  // flat over the batch
@@ -895,6 +897,10 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq
   a.maxseg = plan.maxseg;
   a.pipelined = plan.pipelined;
   a.votes_only = lse_obs ? 1 : 0;
+  if (lse_obs) {  // nothing couples the units any more: one phase over all of them
+    a.upw = plan.units;
+    a.nwaves = 1;
+  }
   a.c2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
   a.partials = partials;
   a.lse2 = lse2;
@@ -904,7 +910,7 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq
   if (lse_obs) {
     const cudaError_t e =
         launch_pdl(lse_prep_kernel, dim3(plan.units), dim3(MAX_COLS), 0, stream, lse_obs, lse2,
-                   counters, plan.units, plan.sub_per_kv, plan.g, plan.hpu, W, plan.ncols);
+                   counters, status, plan.units, plan.sub_per_kv, plan.g, plan.hpu, W, plan.ncols);
     if (e != cudaSuccess) return e;
     *launches += 1;
   }
