@@ -27,7 +27,7 @@ import torch  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries
 # (profiles/): (stage, workload id) -> bytes; None for anything not captured
-NCU_TRAFFIC = {("score", 2): 463.8e6, ("gather", 2): 338.2e6}
+NCU_TRAFFIC = {("score", 2): 463.8e6, ("gather", 2): 338.2e6, ("score-lse", 2): 276.8e6}
 
 METRIC = "prompt_tokens_compressed_per_s"
 UNIT = "prompt tokens/s"
@@ -342,7 +342,7 @@ def main():
                                     "gather": "gather_kernel"}[dom],
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
         "peak_kind": f"of {peak_kind}",
-        "traffic": None if args.lse_in else NCU_TRAFFIC.get((dom, w.wid)),
+        "traffic": NCU_TRAFFIC.get(("score-lse" if args.lse_in and dom == "score" else dom, w.wid)),
         "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": stage_ms[dom],
         "stage_ms_per_layer": stage_ms,
         "whole_step": {"algorithmic_bytes_per_layer": ab["total"], "ms_per_layer": ms_layer,
