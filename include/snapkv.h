@@ -172,6 +172,30 @@ snapkv_status_t snapkv_compress_lse(const void* q_obs, const void* k, const void
                                     void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The whole step (Listing 1) on caches that are not stored as dense [B, Hkv, L, d].
+ * Listing 1 takes key_states / value_states in the framework's [batch, heads, length, d]
+ * order; serving stacks often keep the prompt cache as [B, L, Hkv, d], as one fused K/V
+ * buffer, or as a slice of a larger allocation.  Here k and v are addressed as
+ *   element(b, c, j, t) = base + b * strides[0] + c * strides[1] + j * strides[2] + t
+ * with k_strides / v_strides HOST arrays of three element strides (batch, KV head,
+ * position), read during the call.  Rows of d elements are contiguous.  Every stride must
+ * be positive, a multiple of 8 elements (16 bytes), below 2^39 elements, and the position
+ * stride at least d; otherwise SNAPKV_ERR_INVALID_ARG.  k and v need 16-byte aligned bases
+ * and may have different strides.  lse_obs may be NULL (the normalisers are recomputed,
+ * as in snapkv_compress) or DEVICE fp32 [B, Hq, W] as in snapkv_compress_lse.  q_obs, the
+ * outputs (dense, as in snapkv_compress), the workspace size, errors, ownership and the
+ * results are those of snapkv_compress: the same tiles reach the same arithmetic in the
+ * same order, so the outputs are bit-identical to a call on a dense copy of the cache.
+ */
+snapkv_status_t snapkv_compress_strided(const void* q_obs, const void* k, const void* v,
+                                        const int64_t* k_strides, const int64_t* v_strides,
+                                        const float* lse_obs,
+                                        int B, int Hq, int Hkv, int L, int d, int W,
+                                        int pool_kernel, int pool_type, int budget,
+                                        void* out_k, void* out_v, int32_t* out_idx,
+                                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * snapkv_compress for callers whose tensors live in host memory (pinned memory
  * gives asynchronous copies).  q_obs, k, v, out_k, out_v, out_idx are HOST pointers
  * with the shapes above (out_k/out_v [B,Hq,budget,d], out_idx [B,Hq,budget-W]).

@@ -25,7 +25,7 @@ SYMBOLS = [
     "snapkv_window_scores", "snapkv_pool_topk_workspace_size", "snapkv_pool_topk", "snapkv_gather",
     "snapkv_host_staging_size", "snapkv_compress_host", "snapkv_device_status",
     "snapkv_last_launch_count", "snapkv_pool_topk_static",
-    "snapkv_window_scores_lse", "snapkv_compress_lse",
+    "snapkv_window_scores_lse", "snapkv_compress_lse", "snapkv_compress_strided",
 ]
 
 _lib = None
@@ -60,6 +60,9 @@ def lib() -> ctypes.CDLL:
     L.snapkv_window_scores_lse.argtypes = [c_vp] * 3 + [c_int] * 6 + [c_vp, c_vp, c_sz, c_vp]
     L.snapkv_compress_lse.restype = c_int
     L.snapkv_compress_lse.argtypes = [c_vp] * 4 + [c_int] * 9 + [c_vp] * 3 + [c_vp, c_sz, c_vp]
+    L.snapkv_compress_strided.restype = c_int
+    L.snapkv_compress_strided.argtypes = ([c_vp] * 3 + [ctypes.POINTER(ctypes.c_int64)] * 2 + [c_vp]
+                                          + [c_int] * 9 + [c_vp] * 3 + [c_vp, c_sz, c_vp])
     L.snapkv_pool_topk_workspace_size.restype = c_sz
     L.snapkv_pool_topk_workspace_size.argtypes = [c_int, c_int]
     L.snapkv_pool_topk.restype = c_int
@@ -96,6 +99,13 @@ def _stream_ptr() -> int:
 def _dev_bf16(t: torch.Tensor, name: str) -> torch.Tensor:
     if not (t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()):
         raise SnapKVError(f"{name} must be a contiguous CUDA bf16 tensor")
+    return t
+
+
+def _dev_bf16_rows(t: torch.Tensor, name: str) -> torch.Tensor:
+    """A 4-D [B, Hkv, L, d] view whose rows of d elements are contiguous; the other strides are free."""
+    if not (t.is_cuda and t.dtype == torch.bfloat16 and t.dim() == 4 and t.stride(3) == 1):
+        raise SnapKVError(f"{name} must be a CUDA bf16 [B, Hkv, L, d] view with contiguous rows")
     return t
 
 
@@ -137,9 +147,15 @@ def snapkv_compress(q_obs, k, v, pool_kernel: int, pool_type: int, budget: int,
                     out_k=None, out_v=None, out_idx=None, workspace=None, lse_obs=None):
     """Whole step on device tensors.  Returns (out_k, out_v, out_idx, workspace).
 
+    k, v: bf16 [B, Hkv, L, d], dense or any view of that shape with contiguous rows (strides
+    that are multiples of 8 elements), which goes through snapkv_compress_strided.
+
     out_k/out_v: bf16 [B, Hq, min(budget, L), d]; out_idx: int32 [B, Hq, rows - W].
     """
-    _dev_bf16(q_obs, "q_obs"), _dev_bf16(k, "k"), _dev_bf16(v, "v")
+    _dev_bf16(q_obs, "q_obs"), _dev_bf16_rows(k, "k"), _dev_bf16_rows(v, "v")
+    if tuple(v.shape) != tuple(k.shape):
+        raise SnapKVError("k and v must have the same shape")
+    strided = not (k.is_contiguous() and v.is_contiguous())
     B, Hq, Hkv, L, d, W = _shapes(q_obs, k)
     L_ = lib()
     rows = L_.snapkv_out_rows(L, budget)
@@ -159,7 +175,13 @@ def snapkv_compress(q_obs, k, v, pool_kernel: int, pool_type: int, budget: int,
     tail = (B, Hq, Hkv, L, d, W, pool_kernel, pool_type, eff_budget, out_k.data_ptr(),
             out_v.data_ptr(), out_idx.data_ptr(), workspace.data_ptr(), workspace.numel(),
             _stream_ptr())
-    if lse_obs is None:
+    if strided:
+        # any [B, Hkv, L, d] view with contiguous rows, e.g. a permuted [B, L, Hkv, d] cache
+        st = ctypes.c_int64 * 3
+        code = L_.snapkv_compress_strided(
+            q_obs.data_ptr(), k.data_ptr(), v.data_ptr(), st(*k.stride()[:3]), st(*v.stride()[:3]),
+            None if lse_obs is None else _lse_arg(lse_obs, B, Hq, W), *tail)
+    elif lse_obs is None:
         code = L_.snapkv_compress(q_obs.data_ptr(), k.data_ptr(), v.data_ptr(), *tail)
     else:
         code = L_.snapkv_compress_lse(q_obs.data_ptr(), k.data_ptr(), v.data_ptr(),

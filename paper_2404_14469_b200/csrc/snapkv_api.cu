@@ -169,7 +169,7 @@ static snapkv_status_t window_scores_impl(const void* q_obs, const void* k, cons
     launches = 1;
   }
   cudaError_t e = launch_window_scores(
-      q_obs, k, B, Hq, Hkv, L, d, W, p, out_vote, reinterpret_cast<int*>(ws + w.off_status),
+      q_obs, k, dense_strides(Hkv, L, d), B, Hq, Hkv, L, d, W, p, out_vote, reinterpret_cast<int*>(ws + w.off_status),
       reinterpret_cast<int*>(ws + w.off_counters), reinterpret_cast<float*>(ws + w.off_partials),
       reinterpret_cast<float*>(ws + w.off_lse), s, &launches, lse_obs);
   if (e != cudaSuccess) return SNAPKV_ERR_CUDA;
@@ -220,8 +220,9 @@ snapkv_status_t snapkv_gather(const void* k, const void* v, const int32_t* idx, 
   if (!aligned16(k) || !aligned16(v) || !aligned16(out_k) || !aligned16(out_v))
     return SNAPKV_ERR_INVALID_ARG;
   int launches = 0;
-  cudaError_t e = launch_gather(k, v, idx, B, Hq, Hkv, L, d, W, ksel, ksel + W, out_k, out_v,
-                                static_cast<cudaStream_t>(stream), &launches);
+  const KVStrides ds = dense_strides(Hkv, L, d);
+  cudaError_t e = launch_gather(k, v, ds, ds, idx, B, Hq, Hkv, L, d, W, ksel, ksel + W, out_k,
+                                out_v, static_cast<cudaStream_t>(stream), &launches);
   return e == cudaSuccess ? SNAPKV_OK : SNAPKV_ERR_CUDA;
 }
 
@@ -229,7 +230,9 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
                                      int Hkv, int L, int d, int W, int pool_kernel, int pool_type,
                                      int budget, void* out_k, void* out_v, int32_t* out_idx,
                                      void* workspace, size_t workspace_bytes, void* stream,
-                                     bool keep_status, const float* lse_obs = nullptr) {
+                                     bool keep_status, const float* lse_obs = nullptr,
+                                     const KVStrides* k_str = nullptr,
+                                     const KVStrides* v_str = nullptr) {
   snapkv_status_t st = check_common(B, Hq, Hkv, L, d, W);
   if (st != SNAPKV_OK) return st;
   st = check_pool(pool_kernel, pool_type);
@@ -240,14 +243,16 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
     return SNAPKV_ERR_INVALID_ARG;
   const int n = L - W;
   if (!out_idx && n > 0) return SNAPKV_ERR_INVALID_ARG;
+  const KVStrides ks = k_str ? *k_str : dense_strides(Hkv, L, d);
+  const KVStrides vs = v_str ? *v_str : dense_strides(Hkv, L, d);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int launches = 0;
   if (budget >= L) {
     // Listing 1's early return: nothing is dropped, the cache is expanded to Hq heads.
     if (launch_iota_idx(out_idx, B * Hq, n, budget - W, s, &launches) != cudaSuccess)
       return SNAPKV_ERR_CUDA;
-    if (launch_gather(k, v, nullptr, B, Hq, Hkv, L, d, W, n, budget, out_k, out_v, s, &launches) !=
-        cudaSuccess)
+    if (launch_gather(k, v, ks, vs, nullptr, B, Hq, Hkv, L, d, W, n, budget, out_k, out_v, s,
+                      &launches) != cudaSuccess)
       return SNAPKV_ERR_CUDA;
     g_last_launches = launches;
     return SNAPKV_OK;
@@ -265,7 +270,7 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
   }
   float* vote = reinterpret_cast<float*>(ws + w.off_vote);
   const int ksel = budget - W;
-  if (launch_window_scores(q_obs, k, B, Hq, Hkv, L, d, W, p, vote,
+  if (launch_window_scores(q_obs, k, ks, B, Hq, Hkv, L, d, W, p, vote,
                            reinterpret_cast<int*>(ws + w.off_status),
                            reinterpret_cast<int*>(ws + w.off_counters),
                            reinterpret_cast<float*>(ws + w.off_partials),
@@ -276,8 +281,8 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
                        scratch ? reinterpret_cast<float*>(ws + w.off_pooled) : nullptr, s,
                        &launches) != cudaSuccess)
     return SNAPKV_ERR_CUDA;
-  if (launch_gather(k, v, out_idx, B, Hq, Hkv, L, d, W, ksel, budget, out_k, out_v, s, &launches) !=
-      cudaSuccess)
+  if (launch_gather(k, v, ks, vs, out_idx, B, Hq, Hkv, L, d, W, ksel, budget, out_k, out_v, s,
+                    &launches) != cudaSuccess)
     return SNAPKV_ERR_CUDA;
   g_last_launches = launches;
   return SNAPKV_OK;
@@ -299,6 +304,34 @@ snapkv_status_t snapkv_compress_lse(const void* q_obs, const void* k, const void
   if (!lse_obs || (reinterpret_cast<uintptr_t>(lse_obs) & 3)) return SNAPKV_ERR_INVALID_ARG;
   return compress_impl(q_obs, k, v, B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget, out_k,
                        out_v, out_idx, workspace, workspace_bytes, stream, false, lse_obs);
+}
+
+// One stride triple of snapkv_compress_strided: positive, whole 16-byte vectors, rows of d
+// elements do not overlap, and within what a tensor map can address (byte stride < 2^40).
+static bool strides_ok(const int64_t* st, int d, KVStrides* out) {
+  if (!st) return false;
+  for (int i = 0; i < 3; ++i)
+    if (st[i] <= 0 || (st[i] & 7) != 0 || st[i] >= (1ll << 39)) return false;
+  if (st[2] < d) return false;
+  out->b = st[0];
+  out->h = st[1];
+  out->l = st[2];
+  return true;
+}
+
+snapkv_status_t snapkv_compress_strided(const void* q_obs, const void* k, const void* v,
+                                        const int64_t* k_strides, const int64_t* v_strides,
+                                        const float* lse_obs, int B, int Hq, int Hkv, int L,
+                                        int d, int W, int pool_kernel, int pool_type, int budget,
+                                        void* out_k, void* out_v, int32_t* out_idx,
+                                        void* workspace, size_t workspace_bytes, void* stream) {
+  KVStrides ks, vs;
+  if (!strides_ok(k_strides, d, &ks) || !strides_ok(v_strides, d, &vs))
+    return SNAPKV_ERR_INVALID_ARG;
+  if (lse_obs && (reinterpret_cast<uintptr_t>(lse_obs) & 3)) return SNAPKV_ERR_INVALID_ARG;
+  return compress_impl(q_obs, k, v, B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget, out_k,
+                       out_v, out_idx, workspace, workspace_bytes, stream, false, lse_obs, &ks,
+                       &vs);
 }
 
 size_t snapkv_host_staging_size(int B, int Hq, int Hkv, int L, int d, int W, int pool_kernel,

@@ -32,23 +32,30 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
                : "memory");
 }
 
-// VPR = 16-byte vectors per row.  blockIdx.y is the (batch, query head) pair, blockIdx.x a
-// block of RPB consecutive output rows of that head; one thread moves one vector of K and
-// of V for GATHER_UNROLL rows, all loads issued before the first store.  Index arithmetic
-// is 32-bit except for the final element offsets.
+// Strides of K and of V in 16-byte vectors (batch, KV head, position).
+struct GatherStrides {
+  long long kb, kh, kl, vb, vh, vl;
+};
+
+// VPR = 16-byte vectors per row.  blockIdx.y (+ h0) is the (batch, query head) pair, blockIdx.x
+// a block of RPB consecutive output rows of that head; one thread moves one vector of K and
+// of V for GATHER_UNROLL rows, all loads issued before the first store.
 template <int VPR>
 __global__ void __launch_bounds__(GATHER_THREADS, GATHER_MIN_BLOCKS)
-gather_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v,
-              const int32_t* __restrict__ idx, int g, int L, int W, int ksel, int out_stride,
-              uint4* __restrict__ out_k, uint4* __restrict__ out_v) {
+gather_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v, const GatherStrides st,
+              const int32_t* __restrict__ idx, int h0, int g, int Hkv, int L, int W, int ksel,
+              int out_stride, uint4* __restrict__ out_k, uint4* __restrict__ out_v) {
   constexpr int RPT = GATHER_THREADS / VPR;      // rows covered by the block per unrolled step
   constexpr int RPB = RPT * GATHER_UNROLL;       // rows per block
   const int rows = ksel + W;
   const int n = L - W;
-  const int bh = blockIdx.y;
+  const int bh = h0 + blockIdx.y;
   const int vec = threadIdx.x % VPR;
   const int t0 = blockIdx.x * RPB + threadIdx.x / VPR;
-  const size_t src_head = static_cast<size_t>(bh / g) * L * VPR + vec;
+  const int kvh = bh / g;
+  const int b = kvh / Hkv, c = kvh - b * Hkv;
+  const uint4* k_head = k + (b * st.kb + c * st.kh + vec);
+  const uint4* v_head = v + (b * st.vb + c * st.vh + vec);
   const size_t dst_head = static_cast<size_t>(bh) * out_stride * VPR + vec;
   const int32_t* idx_head = idx ? idx + static_cast<size_t>(bh) * ksel : nullptr;
   int pos[GATHER_UNROLL];
@@ -64,9 +71,8 @@ gather_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v,
 #pragma unroll
   for (int uu = 0; uu < GATHER_UNROLL; ++uu)
     if (ok[uu]) {
-      const size_t src = src_head + static_cast<size_t>(pos[uu]) * VPR;
-      kk[uu] = ld_stream(k + src);
-      vv[uu] = ld_stream(v + src);
+      kk[uu] = ld_stream(k_head + pos[uu] * st.kl);
+      vv[uu] = ld_stream(v_head + pos[uu] * st.vl);
     }
 #pragma unroll
   for (int uu = 0; uu < GATHER_UNROLL; ++uu)
@@ -79,9 +85,10 @@ gather_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v,
 
 }  // namespace
 
-cudaError_t launch_gather(const void* k, const void* v, const int32_t* idx, int B, int Hq, int Hkv,
-                          int L, int d, int W, int ksel, int out_rows_stride, void* out_k,
-                          void* out_v, cudaStream_t stream, int* launches) {
+cudaError_t launch_gather(const void* k, const void* v, const KVStrides& ks, const KVStrides& vs,
+                          const int32_t* idx, int B, int Hq, int Hkv, int L, int d, int W, int ksel,
+                          int out_rows_stride, void* out_k, void* out_v, cudaStream_t stream,
+                          int* launches) {
   const int rows = ksel + W;
   const int vpr = d * 2 / 16;
   const int rpb = GATHER_THREADS / vpr * GATHER_UNROLL;
@@ -92,23 +99,20 @@ cudaError_t launch_gather(const void* k, const void* v, const int32_t* idx, int 
   const uint4* vp = static_cast<const uint4*>(v);
   uint4* okp = static_cast<uint4*>(out_k);
   uint4* ovp = static_cast<uint4*>(out_v);
+  // strides are multiples of 8 elements (the callers check): whole 16-byte vectors
+  const GatherStrides st = {ks.b / 8, ks.h / 8, ks.l / 8, vs.b / 8, vs.h / 8, vs.l / 8};
   const unsigned gx = static_cast<unsigned>((rows + rpb - 1) / rpb);
   // blockIdx.y is limited to 65535: go through the heads in slabs if there are more
-  // (each slab starts on a KV-head boundary so that bh / g stays right inside the kernel)
-  const long long slab = 65535 / g * g > 0 ? 65535 / g * g : g;
+  const long long slab = 65535;
   for (long long h0 = 0; h0 < heads; h0 += slab) {
     const unsigned gy = static_cast<unsigned>(heads - h0 < slab ? heads - h0 : slab);
-    const int32_t* idx_s = idx ? idx + static_cast<size_t>(h0) * ksel : nullptr;
-    uint4* ok_s = okp + static_cast<size_t>(h0) * out_rows_stride * vpr;
-    uint4* ov_s = ovp + static_cast<size_t>(h0) * out_rows_stride * vpr;
-    const uint4* k_s = kp + static_cast<size_t>(h0 / g) * L * vpr;
-    const uint4* v_s = vp + static_cast<size_t>(h0 / g) * L * vpr;
+    const int h0i = static_cast<int>(h0);
     if (vpr == 16)
-      gather_kernel<16><<<dim3(gx, gy), GATHER_THREADS, 0, stream>>>(k_s, v_s, idx_s, g, L, W, ksel,
-                                                                    out_rows_stride, ok_s, ov_s);
+      gather_kernel<16><<<dim3(gx, gy), GATHER_THREADS, 0, stream>>>(
+          kp, vp, st, idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
     else
-      gather_kernel<8><<<dim3(gx, gy), GATHER_THREADS, 0, stream>>>(k_s, v_s, idx_s, g, L, W, ksel,
-                                                                   out_rows_stride, ok_s, ov_s);
+      gather_kernel<8><<<dim3(gx, gy), GATHER_THREADS, 0, stream>>>(
+          kp, vp, st, idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
     *launches += 1;
   }
   return cudaGetLastError();

@@ -46,6 +46,16 @@ struct ScorePlan {
   int pipelined;    // how many waves the statistics pass runs ahead of the vote pass (>= 1)
 };
 
+// Where a K or V tensor's rows are: element strides between consecutive batches, KV heads and
+// positions of a tensor addressed as [batch][KV head][position][d] with d contiguous.  The
+// dense [B, Hkv, L, d] cache of Listing 1 is {Hkv*L*d, L*d, d}.
+struct KVStrides {
+  long long b, h, l;
+};
+inline KVStrides dense_strides(int Hkv, int L, int d) {
+  return KVStrides{static_cast<long long>(Hkv) * L * d, static_cast<long long>(L) * d, d};
+}
+
 struct WorkspaceLayout {
   size_t off_status, off_counters, off_partials, off_lse, off_vote, off_pooled, total;
 };
@@ -60,8 +70,9 @@ size_t select_scratch_bytes(int rows, int n);  // 0 when the rows fit one CTA
 // kernel starts (the callers clear it together with the status block).  With `lse_obs`
 // (device fp32 [B*Hq, W], natural-log sum-exp of every window row) the statistics pass is
 // skipped: a small kernel converts the rows first, then only the vote pass runs.
-cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv, int L,
-                                 int d, int W, const ScorePlan& plan, float* vote, int* status,
+cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrides& ks, int B,
+                                 int Hq, int Hkv, int L, int d, int W, const ScorePlan& plan,
+                                 float* vote, int* status,
                                  int* counters, float* partials, float* lse2, cudaStream_t stream,
                                  int* launches, const float* lse_obs = nullptr);
 
@@ -72,9 +83,10 @@ cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel
                              cudaStream_t stream, int* launches);
 
 // Gather + append.  idx == nullptr copies rows 0..ksel-1 (identity path).
-cudaError_t launch_gather(const void* k, const void* v, const int32_t* idx, int B, int Hq, int Hkv,
-                          int L, int d, int W, int ksel, int out_rows_stride, void* out_k,
-                          void* out_v, cudaStream_t stream, int* launches);
+cudaError_t launch_gather(const void* k, const void* v, const KVStrides& ks, const KVStrides& vs,
+                          const int32_t* idx, int B, int Hq, int Hkv, int L, int d, int W, int ksel,
+                          int out_rows_stride, void* out_k, void* out_v, cudaStream_t stream,
+                          int* launches);
 
 cudaError_t launch_iota_idx(int32_t* out_idx, int rows, int n, int row_stride, cudaStream_t stream,
                             int* launches);

@@ -67,7 +67,7 @@ constexpr int NLB = 8;                // buffers for merged log-sum-exp rows
 constexpr int MERGE_SEGS = 32;        // partials staged in shared memory per merge round
 
 struct ScoreArgs {
-  int L, n, W;
+  int L, n, W, Hkv;
   int hpu, ncols, npad;
   int sub_per_kv, g;
   int units, upw, nwaves;   // units per wave, number of waves
@@ -311,6 +311,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                           sb * 64, qrow0);
         }
         ++nitem;
+        const int kb = ukv / a.Hkv, kh = ukv - kb * a.Hkv;  // the K map is (d, L, Hkv, B)
         const int nt = it.t1 - it.t0;
         for (int k = 0; k < nt; ++k, ++git) {
           const int s = git % STAGES;
@@ -322,9 +323,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           // which keeps the next wave's statistics-pass lines resident instead
           for (int sb = 0; sb < SUBT; ++sb) {
             if (it.vote)
-              tma_load_3d_hint(stage_addr(s, sb), &tmK, bar_full(s), sb * 64, key0, ukv, pol_first);
+              tma_load_4d_hint(stage_addr(s, sb), &tmK, bar_full(s), sb * 64, key0, kh, kb, pol_first);
             else
-              tma_load_3d(stage_addr(s, sb), &tmK, bar_full(s), sb * 64, key0, ukv);
+              tma_load_4d(stage_addr(s, sb), &tmK, bar_full(s), sb * 64, key0, kh, kb);
           }
         }
         return true;
@@ -742,7 +743,7 @@ bool encode_map(CUtensorMap* m, const void* base, int rank, const cuuint64_t* di
                 const cuuint64_t* strides_bytes, const cuuint32_t* box) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
-  cuuint32_t estr[3] = {1, 1, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims,
             strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -862,17 +863,21 @@ bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* pla
   return true;
 }
 
-cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq, int Hkv, int L,
-                                 int d, int W, const ScorePlan& plan, float* vote, int* status,
+cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrides& ks, int B,
+                                 int Hq, int Hkv, int L, int d, int W, const ScorePlan& plan,
+                                 float* vote, int* status,
                                  int* counters, float* partials, float* lse2, cudaStream_t stream,
                                  int* launches, const float* lse_obs) {
   CUtensorMap tmK, tmQ;
   {
-    cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(L),
-                          static_cast<cuuint64_t>(B) * Hkv};
-    cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 2, static_cast<cuuint64_t>(L) * d * 2};
-    cuuint32_t box[3] = {64, TILE_KEYS, 1};
-    if (!encode_map(&tmK, k, 3, dims, strides, box)) return cudaErrorInvalidValue;
+    // (d, position, KV head, batch) with the caller's strides: any layout whose rows of d
+    // elements are contiguous is one tensor map, e.g. [B, L, Hkv, d] as well as [B, Hkv, L, d]
+    cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(L),
+                          static_cast<cuuint64_t>(Hkv), static_cast<cuuint64_t>(B)};
+    cuuint64_t strides[3] = {static_cast<cuuint64_t>(ks.l) * 2, static_cast<cuuint64_t>(ks.h) * 2,
+                             static_cast<cuuint64_t>(ks.b) * 2};
+    cuuint32_t box[4] = {64, TILE_KEYS, 1, 1};
+    if (!encode_map(&tmK, k, 4, dims, strides, box)) return cudaErrorInvalidValue;
   }
   {
     cuuint64_t dims[2] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(B) * Hq * W};
@@ -884,6 +889,7 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, int B, int Hq
   a.L = L;
   a.n = L - W;
   a.W = W;
+  a.Hkv = Hkv;
   a.hpu = plan.hpu;
   a.ncols = plan.ncols;
   a.npad = plan.npad;

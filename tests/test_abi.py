@@ -125,6 +125,25 @@ def test_other_entry_points_reject_bad_arguments(L):
                                  FAKE, None, 0, None) == 3
 
 
+def test_strided_entry_point_checks_its_strides(L):
+    import ctypes
+    st = ctypes.c_int64 * 3
+    dense = st(4 * 1024 * 64, 1024 * 64, 64)
+    args = (None, 1, 4, 4, 1024, 64, 32, 7, 0, 256, FAKE, FAKE, FAKE)
+
+    def call(ks, vs, ws=(FAKE, 1 << 30)):
+        return L.snapkv_compress_strided(FAKE, FAKE, FAKE, ks, vs, *args, ws[0], ws[1], None)
+
+    assert call(None, dense) == 1 and call(dense, None) == 1          # missing stride arrays
+    assert call(st(4 * 1024 * 64, 1024 * 64, 60), dense) == 1         # not whole 16-byte vectors
+    assert call(dense, st(4 * 1024 * 64, 1024 * 64, 56)) == 1         # rows would overlap
+    assert call(st(0, 1024 * 64, 64), dense) == 1                     # zero stride
+    assert call(dense, st(4 * 1024 * 64, -64, 64)) == 1               # negative stride
+    assert call(st(1 << 39, 1024 * 64, 64), dense) == 1               # beyond a tensor map's reach
+    # acceptable strides ([B, L, Hkv, d] order): the next check is the workspace
+    assert call(st(1024 * 4 * 64, 64, 4 * 64), dense, (None, 0)) == 3
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(sk, "_lib", None)
     monkeypatch.setattr(sk, "LIB_PATH", "/nonexistent/libsnapkv.so")
