@@ -32,6 +32,10 @@ A variant outside the paper's listing is stated too: votes_given_lse / window_ls
 lse_obs / compress(lse=...) take the window rows' log-sum-exp as an input (the prompt
 phase's attention kernel holds it) instead of recomputing the softmax.
 
+A second one, for grouped-query attention: group_votes / compress_grouped let the query
+heads of a group select TOGETHER on the KV head they share (Eq. 1's sum runs over the
+window rows of all the group's heads), which keeps the compressed cache at Hkv heads.
+
 Every function here is pinned by tests that do not go through this file's own
 formulas (closed forms, invariants, library routines, brute force): see
 tests/test_oracle_*.py.  Nothing is "parity unpinned".
@@ -273,4 +277,74 @@ def compress(q_obs: np.ndarray, k: np.ndarray, v: np.ndarray, pool_kernel: int,
     else:
         for u in units:
             unit(u)
+    return {"out_k": out_k, "out_v": out_v, "out_idx": out_idx, "vote": vote, "pooled": pooled}
+
+
+def group_votes(vote_heads: np.ndarray) -> np.ndarray:
+    """Shared selection under grouped-query attention: all window queries of all query
+    heads of a group vote on the keys of the KV head they share,
+    C_group[j] = sum over the group's heads h and window rows i of p_h[i, j]
+    (Eq. 1 with the sum extended over the group's heads).  [g, n] -> [n]."""
+    g, n = vote_heads.shape
+    out = np.zeros(n, dtype=np.float64)
+    for h in range(g):
+        out = out + vote_heads[h]
+    return out
+
+
+def compress_grouped(q_obs: np.ndarray, k: np.ndarray, v: np.ndarray, pool_kernel: int,
+                     pool_type: int, budget: int, lse=None, kv_heads=None):
+    """The step with ONE selection per KV head (Listing 1 applied to the KV head with the
+    votes of its whole query group): score and vote per query head as in `compress`, sum the
+    votes over the group (group_votes), then pool, top-k and gather per KV head.
+
+    Returns a dict with
+      out_k, out_v : uint16 [B, Hkv, rows, d], rows = min(budget, L)
+      out_idx      : int64  [B, Hkv, rows - W] ascending prefix positions
+      vote, pooled : fp64   [B, Hkv, n] group votes (None on the identity path)
+    With Hq == Hkv this is `compress`.  `lse` as in `compress`; `kv_heads` optionally
+    restricts the work to a list of (b, c) pairs.
+    """
+    B, Hq, Hkv, L, d, W = _check_shapes(q_obs, k, v)
+    if budget <= W:
+        raise ValueError("budget must exceed the window")
+    n = L - W
+    g = Hq // Hkv
+    if budget >= L:
+        return {
+            "out_k": np.ascontiguousarray(k),
+            "out_v": np.ascontiguousarray(v),
+            "out_idx": np.broadcast_to(np.arange(n, dtype=np.int64), (B, Hkv, n)).copy(),
+            "vote": None,
+            "pooled": None,
+        }
+    ksel = budget - W
+    out_k = np.zeros((B, Hkv, budget, d), dtype=np.uint16)
+    out_v = np.zeros((B, Hkv, budget, d), dtype=np.uint16)
+    out_idx = np.zeros((B, Hkv, ksel), dtype=np.int64)
+    vote = np.zeros((B, Hkv, n), dtype=np.float64)
+    pooled = np.zeros((B, Hkv, n), dtype=np.float64)
+    wanted = None if kv_heads is None else set(kv_heads)
+    for b in range(B):
+        for c in range(Hkv):
+            if wanted is not None and (b, c) not in wanted:
+                continue
+            kf = bf16_bits_to_f64(k[b, c])
+            per_head = np.empty((g, n), dtype=np.float64)
+            for t, h in enumerate(range(c * g, (c + 1) * g)):
+                qf = bf16_bits_to_f64(q_obs[b, h])
+                if lse is None:
+                    per_head[t] = window_votes(qf, kf)
+                else:
+                    per_head[t] = votes_given_lse(window_logits(qf, kf), lse[b, h])
+            vt = group_votes(per_head)
+            pv = pool1d(vt, pool_kernel, pool_type)
+            idx = topk_positions(pv, ksel)
+            vote[b, c] = vt
+            pooled[b, c] = pv
+            out_idx[b, c] = idx
+            out_k[b, c, :ksel] = k[b, c, idx]
+            out_v[b, c, :ksel] = v[b, c, idx]
+            out_k[b, c, ksel:] = k[b, c, n:]
+            out_v[b, c, ksel:] = v[b, c, n:]
     return {"out_k": out_k, "out_v": out_v, "out_idx": out_idx, "vote": vote, "pooled": pooled}
