@@ -45,15 +45,17 @@ def load_peaks():
     return 6650.0, "fallback"
 
 
-def algorithmic_bytes(w, budget):
+def algorithmic_bytes(w, budget, heads_out=None):
     """Per layer: K read once + Q_obs + selected K/V rows read + compressed K/V written +
-    out_idx written (fp32 vote scratch traffic is extra and not counted)."""
+    out_idx written (fp32 vote scratch traffic is extra and not counted).  `heads_out`: heads of
+    the compressed cache (Hq, or Hkv with one selection per KV head)."""
     rows = min(budget, w.L)
     ksel = rows - w.W
+    ho = heads_out or w.Hq
     k_read = w.B * w.Hkv * w.L * w.d * 2
     q_read = w.B * w.Hq * w.W * w.d * 2
-    sel = 2 * w.B * w.Hq * rows * w.d * 2
-    idx = w.B * w.Hq * ksel * 4
+    sel = 2 * w.B * ho * rows * w.d * 2
+    idx = w.B * ho * ksel * 4
     return {"score": k_read + q_read, "gather": 2 * sel + idx, "total": k_read + q_read + 2 * sel + idx}
 
 
@@ -189,6 +191,9 @@ def main():
     ap.add_argument("--lse-in", action="store_true",
                     help="time the supplied-normaliser variant (snapkv_compress_lse): the window "
                          "rows' log-sum-exp is an input, K is swept once; not the paper's path")
+    ap.add_argument("--grouped", action="store_true",
+                    help="time the shared-selection variant (snapkv_compress_grouped): one "
+                         "selection per KV head, the compressed cache keeps Hkv heads")
     args = ap.parse_args()
 
     from paper_2404_14469_b200 import synth
@@ -228,9 +233,10 @@ def main():
     for layer in range(layers):
         d = synth.make_layer(w, layer + replicas.layer_seed_offset(rank), device=str(dev))
         ins.append((d["q_obs"], d["k"], d["v"]))
-    out_k = [torch.empty(w.B, w.Hq, budget, w.d, dtype=torch.bfloat16, device=dev) for _ in range(layers)]
+    ho = w.Hkv if args.grouped else w.Hq
+    out_k = [torch.empty(w.B, ho, budget, w.d, dtype=torch.bfloat16, device=dev) for _ in range(layers)]
     out_v = [torch.empty_like(t) for t in out_k]
-    out_idx = [torch.empty(w.B, w.Hq, ksel, dtype=torch.int32, device=dev) for _ in range(layers)]
+    out_idx = [torch.empty(w.B, ho, ksel, dtype=torch.int32, device=dev) for _ in range(layers)]
     ws = torch.empty(sk.snapkv_workspace_size(w.B, w.Hq, w.Hkv, w.L, w.d, w.W, w.pool_kernel, ptype, budget),
                      dtype=torch.uint8, device=dev)
     vote = torch.empty(w.B * w.Hq, w.n, dtype=torch.float32, device=dev)
@@ -253,7 +259,7 @@ def main():
         for i in range(layers):
             q, k, v = ins[i]
             sk.snapkv_compress(q, k, v, w.pool_kernel, ptype, budget, out_k[i], out_v[i], out_idx[i], ws,
-                               lse_obs=lses[i])
+                               lse_obs=lses[i], grouped=args.grouped)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -295,9 +301,12 @@ def main():
             ev[0].record()
             sk.snapkv_window_scores(q, k, vote.view(w.B, w.Hq, w.n), ws, lse_obs=lses[i])
             ev[1].record()
-            sk.snapkv_pool_topk(vote, w.pool_kernel, ptype, ksel, out_idx[i].view(w.B * w.Hq, ksel), ws)
+            # (the staged select has no group sum: with --grouped only the gather stage, on the
+            # indices the fused call left, and the scoring stage are timed separately)
+            if not args.grouped:
+                sk.snapkv_pool_topk(vote, w.pool_kernel, ptype, ksel, out_idx[i].view(w.B * w.Hq, ksel), ws)
             ev[2].record()
-            lib.snapkv_gather(k.data_ptr(), v.data_ptr(), out_idx[i].data_ptr(), w.B, w.Hq, w.Hkv, w.L,
+            lib.snapkv_gather(k.data_ptr(), v.data_ptr(), out_idx[i].data_ptr(), w.B, ho, w.Hkv, w.L,
                               w.d, w.W, ksel, out_k[i].data_ptr(), out_v[i].data_ptr(),
                               int(torch.cuda.current_stream().cuda_stream))
             ev[3].record()
@@ -328,7 +337,9 @@ def main():
     ms_layer = ms_step / layers
     tokens = w.B * w.L * world
     value = tokens / (ms_step * 1e-3)
-    ab = algorithmic_bytes(w, budget)
+    ab = algorithmic_bytes(w, budget, ho)
+    if args.grouped:
+        stage_ms["select"] = None
     peak, peak_kind = load_peaks()
 
     # roofline of the dominant stage; the gather is one launch per layer, the scoring is a
@@ -353,7 +364,7 @@ def main():
 
     # end to end through the host-buffer entry point: pinned host tensors in, pinned out
     e2e = None
-    if not args.no_e2e and not args.lse_in:
+    if not args.no_e2e and not args.lse_in and not args.grouped:
         q, k, v = (t.cpu().pin_memory() for t in ins[0])
         hk = torch.empty(w.B, w.Hq, budget, w.d, dtype=torch.bfloat16).pin_memory()
         hv = torch.empty_like(hk).pin_memory()
@@ -396,6 +407,10 @@ def main():
         if args.lse_in:
             cfg["variant"] = ("lse-in: the window rows' log-sum-exp is an input, one sweep over K "
                               "(snapkv_compress_lse; not the paper's path)")
+        if args.grouped:
+            cfg["variant"] = (cfg.get("variant", "") + " grouped: one selection per KV head from the "
+                              "group's summed votes, cache of Hkv heads (snapkv_compress_grouped; "
+                              "not the paper's path)").strip()
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,

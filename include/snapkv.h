@@ -196,6 +196,29 @@ snapkv_status_t snapkv_compress_strided(const void* q_obs, const void* k, const 
                                         void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The step with ONE selection per KV head under grouped-query attention, so that the
+ * compressed cache keeps Hkv heads instead of being expanded to Hq.  Listing 1 has a single
+ * num_heads; here Eq. 1's sum over the window queries runs over the window rows of ALL the
+ * query heads of a group: vote_group[b, c, j] = sum over h with kv(h) = c and over window rows
+ * i of softmax_i(q[b,h,i] . k[b,c] / sqrt(d))[j], added in ascending head order in fp32.
+ * Pooling, top-k (Eq. 2) and the gather then run once per KV head:
+ *   out_k/v bf16 [B, Hkv, budget, d], out_idx int32 [B, Hkv, budget - W]  (device)
+ * with the row order, ties and identity rule (budget >= L: rows [0, L) copied per KV head)
+ * of snapkv_compress.  With Hq == Hkv the results are those of snapkv_compress.
+ * k_strides / v_strides: NULL for dense [B, Hkv, L, d], else as in snapkv_compress_strided;
+ * lse_obs: NULL, or DEVICE fp32 [B, Hq, W] as in snapkv_compress_lse.  Workspace size,
+ * errors and ownership as in snapkv_compress (snapkv_workspace_size with the same
+ * arguments: the per-head votes still go through the workspace).
+ */
+snapkv_status_t snapkv_compress_grouped(const void* q_obs, const void* k, const void* v,
+                                        const int64_t* k_strides, const int64_t* v_strides,
+                                        const float* lse_obs,
+                                        int B, int Hq, int Hkv, int L, int d, int W,
+                                        int pool_kernel, int pool_type, int budget,
+                                        void* out_k, void* out_v, int32_t* out_idx,
+                                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * snapkv_compress for callers whose tensors live in host memory (pinned memory
  * gives asynchronous copies).  q_obs, k, v, out_k, out_v, out_idx are HOST pointers
  * with the shapes above (out_k/out_v [B,Hq,budget,d], out_idx [B,Hq,budget-W]).

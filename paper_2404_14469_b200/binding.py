@@ -26,6 +26,7 @@ SYMBOLS = [
     "snapkv_host_staging_size", "snapkv_compress_host", "snapkv_device_status",
     "snapkv_last_launch_count", "snapkv_pool_topk_static",
     "snapkv_window_scores_lse", "snapkv_compress_lse", "snapkv_compress_strided",
+    "snapkv_compress_grouped",
 ]
 
 _lib = None
@@ -63,6 +64,8 @@ def lib() -> ctypes.CDLL:
     L.snapkv_compress_strided.restype = c_int
     L.snapkv_compress_strided.argtypes = ([c_vp] * 3 + [ctypes.POINTER(ctypes.c_int64)] * 2 + [c_vp]
                                           + [c_int] * 9 + [c_vp] * 3 + [c_vp, c_sz, c_vp])
+    L.snapkv_compress_grouped.restype = c_int
+    L.snapkv_compress_grouped.argtypes = L.snapkv_compress_strided.argtypes
     L.snapkv_pool_topk_workspace_size.restype = c_sz
     L.snapkv_pool_topk_workspace_size.argtypes = [c_int, c_int]
     L.snapkv_pool_topk.restype = c_int
@@ -143,8 +146,17 @@ def snapkv_compress_lse(q_obs, k, v, lse_obs, pool_kernel: int, pool_type: int, 
                            workspace, lse_obs=lse_obs)
 
 
+def snapkv_compress_grouped(q_obs, k, v, pool_kernel: int, pool_type: int, budget: int,
+                            out_k=None, out_v=None, out_idx=None, workspace=None, lse_obs=None):
+    """One selection per KV head: the query heads of a group vote together and the cache keeps
+    Hkv heads.  Returns (out_k, out_v [B, Hkv, rows, d], out_idx [B, Hkv, rows - W], workspace)."""
+    return snapkv_compress(q_obs, k, v, pool_kernel, pool_type, budget, out_k, out_v, out_idx,
+                           workspace, lse_obs=lse_obs, grouped=True)
+
+
 def snapkv_compress(q_obs, k, v, pool_kernel: int, pool_type: int, budget: int,
-                    out_k=None, out_v=None, out_idx=None, workspace=None, lse_obs=None):
+                    out_k=None, out_v=None, out_idx=None, workspace=None, lse_obs=None,
+                    grouped: bool = False):
     """Whole step on device tensors.  Returns (out_k, out_v, out_idx, workspace).
 
     k, v: bf16 [B, Hkv, L, d], dense or any view of that shape with contiguous rows (strides
@@ -163,23 +175,26 @@ def snapkv_compress(q_obs, k, v, pool_kernel: int, pool_type: int, budget: int,
     # call it with budget = L so that the tensors stay dense
     eff_budget = rows
     dev = k.device
+    Ho = Hkv if grouped else Hq
     if out_k is None:
-        out_k = torch.empty(B, Hq, rows, d, dtype=torch.bfloat16, device=dev)
+        out_k = torch.empty(B, Ho, rows, d, dtype=torch.bfloat16, device=dev)
     if out_v is None:
-        out_v = torch.empty(B, Hq, rows, d, dtype=torch.bfloat16, device=dev)
+        out_v = torch.empty(B, Ho, rows, d, dtype=torch.bfloat16, device=dev)
     if out_idx is None:
-        out_idx = torch.empty(B, Hq, rows - W, dtype=torch.int32, device=dev)
+        out_idx = torch.empty(B, Ho, rows - W, dtype=torch.int32, device=dev)
     need = L_.snapkv_workspace_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, eff_budget)
     if workspace is None or workspace.numel() < need:
         workspace = _alloc_ws(need, dev)
     tail = (B, Hq, Hkv, L, d, W, pool_kernel, pool_type, eff_budget, out_k.data_ptr(),
             out_v.data_ptr(), out_idx.data_ptr(), workspace.data_ptr(), workspace.numel(),
             _stream_ptr())
-    if strided:
+    if strided or grouped:
         # any [B, Hkv, L, d] view with contiguous rows, e.g. a permuted [B, L, Hkv, d] cache
         st = ctypes.c_int64 * 3
-        code = L_.snapkv_compress_strided(
-            q_obs.data_ptr(), k.data_ptr(), v.data_ptr(), st(*k.stride()[:3]), st(*v.stride()[:3]),
+        fn = L_.snapkv_compress_grouped if grouped else L_.snapkv_compress_strided
+        code = fn(
+            q_obs.data_ptr(), k.data_ptr(), v.data_ptr(),
+            st(*k.stride()[:3]) if strided else None, st(*v.stride()[:3]) if strided else None,
             None if lse_obs is None else _lse_arg(lse_obs, B, Hq, W), *tail)
     elif lse_obs is None:
         code = L_.snapkv_compress(q_obs.data_ptr(), k.data_ptr(), v.data_ptr(), *tail)

@@ -232,7 +232,7 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
                                      void* workspace, size_t workspace_bytes, void* stream,
                                      bool keep_status, const float* lse_obs = nullptr,
                                      const KVStrides* k_str = nullptr,
-                                     const KVStrides* v_str = nullptr) {
+                                     const KVStrides* v_str = nullptr, bool grouped = false) {
   snapkv_status_t st = check_common(B, Hq, Hkv, L, d, W);
   if (st != SNAPKV_OK) return st;
   st = check_pool(pool_kernel, pool_type);
@@ -245,13 +245,17 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
   if (!out_idx && n > 0) return SNAPKV_ERR_INVALID_ARG;
   const KVStrides ks = k_str ? *k_str : dense_strides(Hkv, L, d);
   const KVStrides vs = v_str ? *v_str : dense_strides(Hkv, L, d);
+  // shared selection: the votes of a group's query heads are summed when the select kernel
+  // loads them, and the cache keeps Hkv heads
+  const int Ho = grouped ? Hkv : Hq;
+  const int gsum = grouped ? Hq / Hkv : 1;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int launches = 0;
   if (budget >= L) {
     // Listing 1's early return: nothing is dropped, the cache is expanded to Hq heads.
-    if (launch_iota_idx(out_idx, B * Hq, n, budget - W, s, &launches) != cudaSuccess)
+    if (launch_iota_idx(out_idx, B * Ho, n, budget - W, s, &launches) != cudaSuccess)
       return SNAPKV_ERR_CUDA;
-    if (launch_gather(k, v, ks, vs, nullptr, B, Hq, Hkv, L, d, W, n, budget, out_k, out_v, s,
+    if (launch_gather(k, v, ks, vs, nullptr, B, Ho, Hkv, L, d, W, n, budget, out_k, out_v, s,
                       &launches) != cudaSuccess)
       return SNAPKV_ERR_CUDA;
     g_last_launches = launches;
@@ -277,11 +281,11 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
                            reinterpret_cast<float*>(ws + w.off_lse), s, &launches, lse_obs) !=
       cudaSuccess)
     return SNAPKV_ERR_CUDA;
-  if (launch_pool_topk(vote, B * Hq, n, pool_kernel, pool_type, ksel, out_idx,
+  if (launch_pool_topk(vote, B * Ho, n, pool_kernel, pool_type, ksel, out_idx,
                        scratch ? reinterpret_cast<float*>(ws + w.off_pooled) : nullptr, s,
-                       &launches) != cudaSuccess)
+                       &launches, gsum) != cudaSuccess)
     return SNAPKV_ERR_CUDA;
-  if (launch_gather(k, v, ks, vs, out_idx, B, Hq, Hkv, L, d, W, ksel, budget, out_k, out_v, s,
+  if (launch_gather(k, v, ks, vs, out_idx, B, Ho, Hkv, L, d, W, ksel, budget, out_k, out_v, s,
                     &launches) != cudaSuccess)
     return SNAPKV_ERR_CUDA;
   g_last_launches = launches;
@@ -332,6 +336,21 @@ snapkv_status_t snapkv_compress_strided(const void* q_obs, const void* k, const 
   return compress_impl(q_obs, k, v, B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget, out_k,
                        out_v, out_idx, workspace, workspace_bytes, stream, false, lse_obs, &ks,
                        &vs);
+}
+
+snapkv_status_t snapkv_compress_grouped(const void* q_obs, const void* k, const void* v,
+                                        const int64_t* k_strides, const int64_t* v_strides,
+                                        const float* lse_obs, int B, int Hq, int Hkv, int L,
+                                        int d, int W, int pool_kernel, int pool_type, int budget,
+                                        void* out_k, void* out_v, int32_t* out_idx,
+                                        void* workspace, size_t workspace_bytes, void* stream) {
+  KVStrides ks, vs;
+  if ((k_strides && !strides_ok(k_strides, d, &ks)) || (v_strides && !strides_ok(v_strides, d, &vs)))
+    return SNAPKV_ERR_INVALID_ARG;
+  if (lse_obs && (reinterpret_cast<uintptr_t>(lse_obs) & 3)) return SNAPKV_ERR_INVALID_ARG;
+  return compress_impl(q_obs, k, v, B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget, out_k,
+                       out_v, out_idx, workspace, workspace_bytes, stream, false, lse_obs,
+                       k_strides ? &ks : nullptr, v_strides ? &vs : nullptr, true);
 }
 
 size_t snapkv_host_staging_size(int B, int Hq, int Hkv, int L, int d, int W, int pool_kernel,

@@ -77,10 +77,12 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrid
                                  int* launches, const float* lse_obs = nullptr);
 
 // Pool + top-k over `rows` rows of fp32 votes.  `pooled_scratch` (select_scratch_bytes bytes)
-// is only touched when select_needs_scratch(n).
+// is only touched when select_needs_scratch(n).  With gsum > 1 a selection row is the sum of
+// gsum consecutive rows of `vote` (which then holds rows * gsum rows): the query heads of a
+// group selecting together.
 cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel, int pool_type,
                              int ksel, int32_t* out_idx, float* pooled_scratch,
-                             cudaStream_t stream, int* launches);
+                             cudaStream_t stream, int* launches, int gsum = 1);
 
 // Gather + append.  idx == nullptr copies rows 0..ksel-1 (identity path).
 cudaError_t launch_gather(const void* k, const void* v, const KVStrides& ks, const KVStrides& vs,

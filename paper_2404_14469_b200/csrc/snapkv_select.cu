@@ -58,9 +58,18 @@ __device__ __forceinline__ int block_exclusive_scan(int x, int* warp_sums_s, int
   return warp_sums_s[warp] + inc - x;
 }
 
+// Vote of position j of a selection row.  With shared selection under grouped-query
+// attention `gsum` consecutive per-head rows of n votes select together: their sum, taken in
+// ascending head order (gsum = 1: the row itself).  `vrow` is the first of those rows.
+__device__ __forceinline__ float ld_vote(const float* __restrict__ vrow, int j, int n, int gsum) {
+  float x = __ldg(vrow + j);
+  for (int t = 1; t < gsum; ++t) x += __ldg(vrow + static_cast<size_t>(t) * n + j);
+  return x;
+}
+
 __global__ void __launch_bounds__(SEL_THREADS, 1)
-pool_topk_kernel(const float* __restrict__ vote, int n, int pool_kernel, int pool_type, int ksel,
-                 int32_t* __restrict__ out_idx, uint32_t* __restrict__ key_scratch) {
+pool_topk_kernel(const float* __restrict__ vote, int n, int gsum, int pool_kernel, int pool_type,
+                 int ksel, int32_t* __restrict__ out_idx, uint32_t* __restrict__ key_scratch) {
   extern __shared__ uint32_t keys_smem[];
   __shared__ int hist[NBINS];
   __shared__ int warp_sums[SEL_WARPS];
@@ -69,7 +78,7 @@ pool_topk_kernel(const float* __restrict__ vote, int n, int pool_kernel, int poo
   __shared__ int wgt[SEL_WARPS], weq[SEL_WARPS];
 
   const int row = blockIdx.x;
-  const float* vrow = vote + static_cast<size_t>(row) * n;
+  const float* vrow = vote + static_cast<size_t>(row) * gsum * n;
   uint32_t* keys = key_scratch ? key_scratch + static_cast<size_t>(row) * n : keys_smem;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int r = pool_kernel >> 1;
@@ -79,11 +88,11 @@ pool_topk_kernel(const float* __restrict__ vote, int n, int pool_kernel, int poo
     const int lo = max(0, j - r), hi = min(n - 1, j + r);
     float p;
     if (pool_type == 0) {
-      p = __ldg(vrow + lo);
-      for (int t = lo + 1; t <= hi; ++t) p = fmaxf(p, __ldg(vrow + t));
+      p = ld_vote(vrow, lo, n, gsum);
+      for (int t = lo + 1; t <= hi; ++t) p = fmaxf(p, ld_vote(vrow, t, n, gsum));
     } else {
       p = 0.f;
-      for (int t = lo; t <= hi; ++t) p += __ldg(vrow + t);
+      for (int t = lo; t <= hi; ++t) p += ld_vote(vrow, t, n, gsum);
       p = p / static_cast<float>(pool_kernel);
     }
     keys[j] = float_to_key(p);
@@ -199,8 +208,8 @@ constexpr int MASK_WORDS = 2;    // a thread owns at most 64 positions (SEL_SMEM
 // (avg): the radius is exactly RMAX, so the window loop has no per-element tests.
 template <int RMAX, int PT>
 __global__ void __launch_bounds__(SEL_THREADS, 1)
-pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_type, int ept,
-                      int ksel, int32_t* __restrict__ out_idx) {
+pool_topk_fast_kernel(const float* __restrict__ vote, int n, int gsum, int r, int pool_type,
+                      int ept, int ksel, int32_t* __restrict__ out_idx) {
   extern __shared__ __align__(16) uint32_t keys[];
   __shared__ int hist[NBINS];
   __shared__ int warp_sums[SEL_WARPS];
@@ -211,7 +220,7 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
   int ncand = 0;
 
   const int row = blockIdx.x;
-  const float* vrow = vote + static_cast<size_t>(row) * n;
+  const float* vrow = vote + static_cast<size_t>(row) * gsum * n;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int base = threadIdx.x * ept;
 
@@ -222,8 +231,29 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int r, int pool_typ
   uint32_t kmin = 0xffffffffu, kmax = 0u;
   {
     const int total = SEL_THREADS * ept;
-    for (int j = threadIdx.x; j < total; j += SEL_THREADS)
-      keys[key_slot4(j)] = (j < n) ? __float_as_uint(__ldg(vrow + j)) : 0u;
+    if (gsum == 1) {
+      for (int j = threadIdx.x; j < total; j += SEL_THREADS)
+        keys[key_slot4(j)] = (j < n) ? __float_as_uint(__ldg(vrow + j)) : 0u;
+    } else {
+      // group sum: four positions per thread and step, so that the loads of a step are
+      // independent of one another; heads are added in ascending order
+      for (int j0 = threadIdx.x; j0 < total; j0 += 4 * SEL_THREADS) {
+        float x[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int t = 0; t < gsum; ++t) {
+          const float* src = vrow + static_cast<size_t>(t) * n;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int j = j0 + u * SEL_THREADS;
+            if (j < n) x[u] += __ldg(src + j);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int j = j0 + u * SEL_THREADS;
+          if (j < total) keys[key_slot4(j)] = __float_as_uint(x[u]);
+        }
+      }
+    }
     __syncthreads();
     // a[]: the last RMAX values before the current block of 8, the block, the next block
     float a[RMAX + 16];
@@ -493,16 +523,17 @@ __device__ __forceinline__ void wide_histogram(const uint32_t (&key_of_thread)[3
 // Pooling of one chunk (staged through shared memory with its halo), keys to scratch, and
 // the first histogram pass.
 __global__ void __launch_bounds__(WIDE_THREADS)
-wide_pool_kernel(const float* __restrict__ vote, int n, int pool_kernel, int pool_type, WideBufs wb) {
+wide_pool_kernel(const float* __restrict__ vote, int n, int gsum, int pool_kernel, int pool_type,
+                 WideBufs wb) {
   __shared__ float raw[WIDE_CHUNK + 2 * WIDE_HALO + (WIDE_CHUNK + 2 * WIDE_HALO) / 32 + 1];
   __shared__ int hist_s[NBINS];
   const int row = blockIdx.y;
   const int c0 = blockIdx.x * WIDE_CHUNK;
   const int r = pool_kernel >> 1;
-  const float* vrow = vote + static_cast<size_t>(row) * n;
+  const float* vrow = vote + static_cast<size_t>(row) * gsum * n;
   for (int t = threadIdx.x; t < WIDE_CHUNK + 2 * r; t += WIDE_THREADS) {
     const int j = c0 - r + t;
-    raw[key_slot(t)] = (j >= 0 && j < n) ? __ldg(vrow + j) : 0.f;
+    raw[key_slot(t)] = (j >= 0 && j < n) ? (gsum == 1 ? __ldg(vrow + j) : ld_vote(vrow, j, n, gsum)) : 0.f;
   }
   __syncthreads();
   uint32_t mine[WIDE_EPT];
@@ -712,7 +743,7 @@ size_t select_scratch_bytes(int rows, int n) {
 
 cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel, int pool_type,
                              int ksel, int32_t* out_idx, float* pooled_scratch,
-                             cudaStream_t stream, int* launches) {
+                             cudaStream_t stream, int* launches, int gsum) {
   static bool attr_done = false;
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(pool_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -733,8 +764,8 @@ cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel
     const int ept = (((n + SEL_THREADS - 1) / SEL_THREADS) + 7) & ~7;
     const int words = key_slot4_host(SEL_THREADS * ept) + 4;
 #define SNAPKV_FAST_LAUNCH(RM, P)                                                            \
-  pool_topk_fast_kernel<RM, P><<<rows, SEL_THREADS, words * 4, stream>>>(vote, n, r, pool_type, \
-                                                                        ept, ksel, out_idx)
+  pool_topk_fast_kernel<RM, P><<<rows, SEL_THREADS, words * 4, stream>>>(vote, n, gsum, r,    \
+                                                                        pool_type, ept, ksel, out_idx)
     // the paper's kernel sizes 5, 7 and 13 have instantiations of their own
     const bool mx = pool_type == 0;
     if (r == 2) { if (mx) SNAPKV_FAST_LAUNCH(2, 0); else SNAPKV_FAST_LAUNCH(2, 1); }
@@ -748,7 +779,7 @@ cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel
   }
   if (!select_needs_scratch(n)) {  // fits one CTA, but the radius is beyond the fast path
     pool_topk_kernel<<<rows, SEL_THREADS, static_cast<size_t>(n) * 4, stream>>>(
-        vote, n, pool_kernel, pool_type, ksel, out_idx, nullptr);
+        vote, n, gsum, pool_kernel, pool_type, ksel, out_idx, nullptr);
     *launches += 1;
     return cudaGetLastError();
   }
@@ -767,7 +798,7 @@ cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel
   cudaError_t e = cudaMemsetAsync(wb.hist, 0, up256(nr * NBINS * 4), stream);
   if (e != cudaSuccess) return e;
   const dim3 grid(wb.nblk, rows);
-  wide_pool_kernel<<<grid, WIDE_THREADS, 0, stream>>>(vote, n, pool_kernel, pool_type, wb);
+  wide_pool_kernel<<<grid, WIDE_THREADS, 0, stream>>>(vote, n, gsum, pool_kernel, pool_type, wb);
   wide_pick_kernel<<<rows, SEL_THREADS, 0, stream>>>(0, ksel, wb);
   wide_hist_kernel<<<grid, WIDE_THREADS, 0, stream>>>(n, 1, wb);
   wide_pick_kernel<<<rows, SEL_THREADS, 0, stream>>>(1, ksel, wb);
@@ -837,6 +868,6 @@ extern "C" snapkv_status_t snapkv_pool_topk_static(const float* vote, int rows, 
   // Every key the kernel reads was written by the same launch, so nothing has to be
   // cleared between calls; whatever the previous call left behind is overwritten or unused.
   pool_topk_kernel<<<rows, SEL_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
-      vote, n, pool_kernel, pool_type, ksel, out_idx, keys);
+      vote, n, 1, pool_kernel, pool_type, ksel, out_idx, keys);
   return cudaGetLastError() == cudaSuccess ? SNAPKV_OK : SNAPKV_ERR_CUDA;
 }
