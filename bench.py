@@ -27,7 +27,7 @@ import torch  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries
 # (profiles/): (stage, workload id) -> bytes; None for anything not captured
-NCU_TRAFFIC = {("score", 2): 463.8e6, ("gather", 2): 338.2e6, ("score-lse", 2): 276.8e6}
+NCU_TRAFFIC = {("score", 2): 464.6e6, ("gather", 2): 338.7e6, ("score-lse", 2): 275.9e6}
 
 METRIC = "prompt_tokens_compressed_per_s"
 UNIT = "prompt tokens/s"
