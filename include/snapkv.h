@@ -219,6 +219,37 @@ snapkv_status_t snapkv_compress_grouped(const void* q_obs, const void* k, const 
                                         void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The whole step (Listing 1) on a batch whose prompts differ in length.  Listing 1 has one
+ * q_len for the batch; the sequences are independent of one another (Sec. 4.1), so each is
+ * compressed as a single-sequence step of its own length, one after the other on `stream`.
+ *   seq_lens       HOST int32 [B]: L_b, W <= L_b <= Lmax.  Sequence b's window is its last W
+ *                  positions, its prefix the L_b - W before them.
+ *   k, v           as in snapkv_compress_strided (k_strides / v_strides NULL: dense
+ *                  [B, Hkv, Lmax, d], each sequence's rows at positions [0, L_b)).
+ *   k_seq_offsets / v_seq_offsets  HOST int64 [B] or NULL: element offset of sequence b's
+ *                  position 0 of KV head 0 from the base pointer (multiples of 8, >= 0); NULL
+ *                  means b * strides[0].  With offsets = Hkv * d * (tokens before b) and
+ *                  strides {any, d, Hkv * d} this reads a packed [total_tokens, Hkv, d] cache.
+ *   q_obs          bf16 [B, Hq, W, d]: each sequence's own last W queries.
+ *   lse_obs        NULL or DEVICE fp32 [B, Hq, W] (as in snapkv_compress_lse, per sequence).
+ *   out_k/v        bf16 [B, Hq, budget, d], out_idx int32 [B, Hq, budget - W] (device).
+ *                  A sequence with budget >= L_b is copied through as in snapkv_compress: rows
+ *                  [0, L_b) written, out_idx[b, :, 0:L_b - W] = 0.., the rest left untouched.
+ * The host arrays are read during the call.  All sequences are validated before anything is
+ * launched (SNAPKV_ERR_INVALID_ARG; SNAPKV_ERR_WORKSPACE if the workspace is smaller than the
+ * largest snapkv_workspace_size(1, Hq, Hkv, L_b, ...) over the sequences with L_b > budget);
+ * the status block keeps the first error of any sequence.  Each sequence's result is that of snapkv_compress on that sequence alone.
+ */
+snapkv_status_t snapkv_compress_varlen(const void* q_obs, const void* k, const void* v,
+                                       const int64_t* k_strides, const int64_t* v_strides,
+                                       const int64_t* k_seq_offsets, const int64_t* v_seq_offsets,
+                                       const int32_t* seq_lens, const float* lse_obs,
+                                       int B, int Hq, int Hkv, int Lmax, int d, int W,
+                                       int pool_kernel, int pool_type, int budget,
+                                       void* out_k, void* out_v, int32_t* out_idx,
+                                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * snapkv_compress for callers whose tensors live in host memory (pinned memory
  * gives asynchronous copies).  q_obs, k, v, out_k, out_v, out_idx are HOST pointers
  * with the shapes above (out_k/out_v [B,Hq,budget,d], out_idx [B,Hq,budget-W]).

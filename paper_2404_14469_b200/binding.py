@@ -26,7 +26,7 @@ SYMBOLS = [
     "snapkv_host_staging_size", "snapkv_compress_host", "snapkv_device_status",
     "snapkv_last_launch_count", "snapkv_pool_topk_static",
     "snapkv_window_scores_lse", "snapkv_compress_lse", "snapkv_compress_strided",
-    "snapkv_compress_grouped",
+    "snapkv_compress_grouped", "snapkv_compress_varlen",
 ]
 
 _lib = None
@@ -66,6 +66,10 @@ def lib() -> ctypes.CDLL:
                                           + [c_int] * 9 + [c_vp] * 3 + [c_vp, c_sz, c_vp])
     L.snapkv_compress_grouped.restype = c_int
     L.snapkv_compress_grouped.argtypes = L.snapkv_compress_strided.argtypes
+    p64, p32 = ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int32)
+    L.snapkv_compress_varlen.restype = c_int
+    L.snapkv_compress_varlen.argtypes = ([c_vp] * 3 + [p64] * 4 + [p32, c_vp] + [c_int] * 9 + [c_vp] * 3
+                                         + [c_vp, c_sz, c_vp])
     L.snapkv_pool_topk_workspace_size.restype = c_sz
     L.snapkv_pool_topk_workspace_size.argtypes = [c_int, c_int]
     L.snapkv_pool_topk.restype = c_int
@@ -202,6 +206,50 @@ def snapkv_compress(q_obs, k, v, pool_kernel: int, pool_type: int, budget: int,
         code = L_.snapkv_compress_lse(q_obs.data_ptr(), k.data_ptr(), v.data_ptr(),
                                       _lse_arg(lse_obs, B, Hq, W), *tail)
     _check(code, "snapkv_compress")
+    return out_k, out_v, out_idx, workspace
+
+
+def snapkv_compress_varlen(q_obs, k, v, seq_lens, pool_kernel: int, pool_type: int, budget: int,
+                           cu_seqlens=None, lse_obs=None, workspace=None):
+    """Batch of prompts of different lengths.  seq_lens: list of B lengths.
+
+    k, v: either a [B, Hkv, Lmax, d] view with contiguous rows (sequence b at positions
+    [0, seq_lens[b])), or, with `cu_seqlens` (list of B starting tokens), a packed
+    [total_tokens, Hkv, d] tensor.  Returns (out_k, out_v [B, Hq, budget, d] zero-filled,
+    out_idx [B, Hq, budget - W] filled with -1, workspace); a sequence with budget >= its
+    length fills only its first rows.
+    """
+    _dev_bf16(q_obs, "q_obs")
+    B, Hq, W, d = q_obs.shape
+    lens = [int(x) for x in seq_lens]
+    st = ctypes.c_int64 * 3
+    if cu_seqlens is None:
+        _dev_bf16_rows(k, "k"), _dev_bf16_rows(v, "v")
+        Hkv, Lmax = k.shape[1], k.shape[2]
+        ks, vs, ko, vo = st(*k.stride()[:3]), st(*v.stride()[:3]), None, None
+    else:
+        if not (k.is_cuda and k.dtype == torch.bfloat16 and k.dim() == 3 and k.is_contiguous()
+                and v.shape == k.shape and v.is_contiguous() and v.dtype == torch.bfloat16):
+            raise SnapKVError("packed k and v must be contiguous CUDA bf16 [total_tokens, Hkv, d]")
+        Hkv, Lmax = k.shape[1], max(lens)
+        row = Hkv * d
+        ks = vs = st(row * 8, d, row)       # the batch stride is not used: offsets are given
+        ko = vo = (ctypes.c_int64 * B)(*[int(c) * row for c in cu_seqlens])
+    L_ = lib()
+    dev = k.device
+    out_k = torch.zeros(B, Hq, budget, d, dtype=torch.bfloat16, device=dev)
+    out_v = torch.zeros_like(out_k)
+    out_idx = torch.full((B, Hq, budget - W), -1, dtype=torch.int32, device=dev)
+    need = max([L_.snapkv_workspace_size(1, Hq, Hkv, x, d, W, pool_kernel, pool_type, budget)
+                for x in set(lens) if x > budget] + [256])
+    if workspace is None or workspace.numel() < need:
+        workspace = _alloc_ws(need, dev)
+    code = L_.snapkv_compress_varlen(
+        q_obs.data_ptr(), k.data_ptr(), v.data_ptr(), ks, vs, ko, vo, (ctypes.c_int32 * B)(*lens),
+        None if lse_obs is None else _lse_arg(lse_obs, B, Hq, W), B, Hq, Hkv, Lmax, d, W,
+        pool_kernel, pool_type, budget, out_k.data_ptr(), out_v.data_ptr(), out_idx.data_ptr(),
+        workspace.data_ptr(), workspace.numel(), _stream_ptr())
+    _check(code, "snapkv_compress_varlen")
     return out_k, out_v, out_idx, workspace
 
 

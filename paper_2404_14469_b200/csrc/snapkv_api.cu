@@ -353,6 +353,58 @@ snapkv_status_t snapkv_compress_grouped(const void* q_obs, const void* k, const 
                        k_strides ? &ks : nullptr, v_strides ? &vs : nullptr, true);
 }
 
+snapkv_status_t snapkv_compress_varlen(const void* q_obs, const void* k, const void* v,
+                                       const int64_t* k_strides, const int64_t* v_strides,
+                                       const int64_t* k_seq_offsets, const int64_t* v_seq_offsets,
+                                       const int32_t* seq_lens, const float* lse_obs, int B,
+                                       int Hq, int Hkv, int Lmax, int d, int W, int pool_kernel,
+                                       int pool_type, int budget, void* out_k, void* out_v,
+                                       int32_t* out_idx, void* workspace, size_t workspace_bytes,
+                                       void* stream) {
+  snapkv_status_t st = check_common(B, Hq, Hkv, Lmax, d, W);
+  if (st != SNAPKV_OK) return st;
+  if (!seq_lens || budget <= W || !q_obs || !k || !v || !out_k || !out_v)
+    return SNAPKV_ERR_INVALID_ARG;
+  KVStrides ks = dense_strides(Hkv, Lmax, d), vs = ks;
+  if ((k_strides && !strides_ok(k_strides, d, &ks)) || (v_strides && !strides_ok(v_strides, d, &vs)))
+    return SNAPKV_ERR_INVALID_ARG;
+  if (lse_obs && (reinterpret_cast<uintptr_t>(lse_obs) & 3)) return SNAPKV_ERR_INVALID_ARG;
+  // every sequence is checked before the first launch
+  for (int b = 0; b < B; ++b) {
+    if (seq_lens[b] < W || seq_lens[b] > Lmax) return SNAPKV_ERR_INVALID_ARG;
+    if (k_seq_offsets && (k_seq_offsets[b] < 0 || (k_seq_offsets[b] & 7))) return SNAPKV_ERR_INVALID_ARG;
+    if (v_seq_offsets && (v_seq_offsets[b] < 0 || (v_seq_offsets[b] & 7))) return SNAPKV_ERR_INVALID_ARG;
+  }
+  for (int b = 0; b < B; ++b) {
+    if (budget >= seq_lens[b]) continue;  // copied through: no scratch
+    const size_t need =
+        snapkv_workspace_size(1, Hq, Hkv, seq_lens[b], d, W, pool_kernel, pool_type, budget);
+    if (need == 0) return SNAPKV_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < need) return SNAPKV_ERR_WORKSPACE;
+  }
+  const size_t head_rows = static_cast<size_t>(Hq) * budget * d * 2;  // bytes of one sequence's out_k
+  int launches = 0;
+  for (int b = 0; b < B; ++b) {
+    const long long ko = k_seq_offsets ? k_seq_offsets[b] : b * ks.b;
+    const long long vo = v_seq_offsets ? v_seq_offsets[b] : b * vs.b;
+    // the sequences are independent (Sec. 4.1): one single-sequence step each, on the same
+    // stream and workspace; the status block keeps the first error of any of them
+    st = compress_impl(static_cast<const uint8_t*>(q_obs) + static_cast<size_t>(b) * Hq * W * d * 2,
+                       static_cast<const uint8_t*>(k) + ko * 2,
+                       static_cast<const uint8_t*>(v) + vo * 2, 1, Hq, Hkv, seq_lens[b], d, W,
+                       pool_kernel, pool_type, budget,
+                       static_cast<uint8_t*>(out_k) + b * head_rows,
+                       static_cast<uint8_t*>(out_v) + b * head_rows,
+                       out_idx ? out_idx + static_cast<size_t>(b) * Hq * (budget - W) : nullptr,
+                       workspace, workspace_bytes, stream, b > 0,
+                       lse_obs ? lse_obs + static_cast<size_t>(b) * Hq * W : nullptr, &ks, &vs);
+    if (st != SNAPKV_OK) return st;
+    launches += g_last_launches;
+  }
+  g_last_launches = launches;
+  return SNAPKV_OK;
+}
+
 size_t snapkv_host_staging_size(int B, int Hq, int Hkv, int L, int d, int W, int pool_kernel,
                                 int pool_type, int budget) {
   if (check_common(B, Hq, Hkv, L, d, W) != SNAPKV_OK) return 0;

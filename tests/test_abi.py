@@ -144,6 +144,24 @@ def test_strided_entry_point_checks_its_strides(L):
     assert call(st(1024 * 4 * 64, 64, 4 * 64), dense, (None, 0)) == 3
 
 
+def test_varlen_entry_point_checks_every_sequence_before_launching(L):
+    import ctypes
+    i32, i64 = ctypes.c_int32 * 3, ctypes.c_int64 * 3
+    tail = (None, 3, 4, 4, 1024, 64, 32, 7, 0, 256, FAKE, FAKE, FAKE)
+
+    def call(lens, koff=None, ws=(FAKE, 1 << 30)):
+        return L.snapkv_compress_varlen(FAKE, FAKE, FAKE, None, None, koff, None, lens, *tail,
+                                        ws[0], ws[1], None)
+
+    assert call(None) == 1                                  # no lengths
+    assert call(i32(1024, 31, 500)) == 1                    # shorter than the window
+    assert call(i32(1024, 1025, 500)) == 1                  # longer than Lmax
+    assert call(i32(1024, 600, 500), i64(0, 4, 64)) == 1    # offset not a whole 16-byte vector
+    assert call(i32(1024, 600, 500), i64(0, -8, 64)) == 1
+    assert call(i32(1024, 600, 500), None, (None, 0)) == 3  # some sequence needs scratch
+    assert call(i32(1024, 600, 500), None, (FAKE, 1024)) == 3
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(sk, "_lib", None)
     monkeypatch.setattr(sk, "LIB_PATH", "/nonexistent/libsnapkv.so")
