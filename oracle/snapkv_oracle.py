@@ -36,6 +36,8 @@ A second one, for grouped-query attention: group_votes / compress_grouped let th
 heads of a group select TOGETHER on the KV head they share (Eq. 1's sum runs over the
 window rows of all the group's heads), which keeps the compressed cache at Hkv heads.
 
+hit_counts / hit_rate state the paper's hit-rate measure of a selection (Sec. 3, Eq. 3-7).
+
 Every function here is pinned by tests that do not go through this file's own
 formulas (closed forms, invariants, library routines, brute force): see
 tests/test_oracle_*.py.  Nothing is "parity unpinned".
@@ -348,3 +350,25 @@ def compress_grouped(q_obs: np.ndarray, k: np.ndarray, v: np.ndarray, pool_kerne
             out_k[b, c, ksel:] = k[b, c, n:]
             out_v[b, c, ksel:] = v[b, c, n:]
     return {"out_k": out_k, "out_v": out_v, "out_idx": out_idx, "vote": vote, "pooled": pooled}
+
+
+def hit_counts(a_cur: np.ndarray, idx: np.ndarray, theta) -> np.ndarray:
+    """Sec. 3, Eq. 3-7 per head: a_cur fp32 [N, L_prefix] (attention of one generated query over
+    the prefix keys), idx int [N, k] (positions chosen by the vote).  Builds the two masks of
+    the definition, M_vote_obs (ones at idx) and M_threshold_cur (a_cur > theta, compared in
+    fp32 as given), and returns int64 [N, 2]: per head the overlap sum(O) and sum(M_threshold_cur).
+    """
+    a = np.asarray(a_cur, dtype=np.float32)
+    N, n = a.shape
+    m_vote = np.zeros((N, n), dtype=bool)
+    for h in range(N):
+        m_vote[h, np.asarray(idx[h], dtype=np.int64)] = True
+    m_thr = a > np.float32(theta)
+    overlap = np.logical_and(m_thr, m_vote)
+    return np.stack([overlap.sum(axis=1), m_thr.sum(axis=1)], axis=1).astype(np.int64)
+
+
+def hit_rate(a_cur: np.ndarray, idx: np.ndarray, theta) -> float:
+    """Eq. 7: H = sum(O) / sum(M_threshold_cur) over all heads (nan when nothing is important)."""
+    c = hit_counts(a_cur, idx, theta)
+    return float(c[:, 0].sum()) / float(c[:, 1].sum()) if c[:, 1].sum() > 0 else float("nan")
