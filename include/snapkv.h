@@ -275,6 +275,20 @@ snapkv_status_t snapkv_compress_host(const void* q_obs, const void* k, const voi
                                      void* staging, size_t staging_bytes, void* stream);
 
 /*
+ * Hit rate of a selection (Sec. 3, Eq. 3-7).  a_cur fp32 [rows, n] device: the attention
+ * features of one generated query over the n prefix keys, one row per head; idx int32
+ * [rows, k] device: the positions the vote selected (distinct within a row; entries outside
+ * [0, n) are ignored); theta: the importance threshold, compared in fp32 with a strict >
+ * (Eq. 5).  Writes out_counts int32 [rows, 2] device: per head {sum of O (Eq. 6: selected
+ * positions whose feature exceeds theta), sum of M_threshold_cur (features exceeding theta)}.
+ * H of Eq. 7 is the ratio of the column sums; the per-row ratios are the per-head rates.
+ * Integer counting: exact, independent of scheduling.  Enqueued on `stream` (a clear of
+ * out_counts, then one kernel); no workspace.  rows <= 65535.
+ */
+snapkv_status_t snapkv_hit_counts(const float* a_cur, const int32_t* idx, int rows, int n, int k,
+                                  float theta, int32_t* out_counts, void* stream);
+
+/*
  * Synchronises `stream`, reads the status word the kernels keep at the start of
  * `workspace` and returns it (SNAPKV_OK or SNAPKV_ERR_TIMEOUT), or SNAPKV_ERR_CUDA
  * if the stream reports an error.  `detail`, if not NULL, receives a code telling

@@ -27,6 +27,7 @@ SYMBOLS = [
     "snapkv_last_launch_count", "snapkv_pool_topk_static",
     "snapkv_window_scores_lse", "snapkv_compress_lse", "snapkv_compress_strided",
     "snapkv_compress_grouped", "snapkv_compress_varlen",
+    "snapkv_hit_counts",
 ]
 
 _lib = None
@@ -70,6 +71,8 @@ def lib() -> ctypes.CDLL:
     L.snapkv_compress_varlen.restype = c_int
     L.snapkv_compress_varlen.argtypes = ([c_vp] * 3 + [p64] * 4 + [p32, c_vp] + [c_int] * 9 + [c_vp] * 3
                                          + [c_vp, c_sz, c_vp])
+    L.snapkv_hit_counts.restype = c_int
+    L.snapkv_hit_counts.argtypes = [c_vp, c_vp, c_int, c_int, c_int, ctypes.c_float, c_vp, c_vp]
     L.snapkv_pool_topk_workspace_size.restype = c_sz
     L.snapkv_pool_topk_workspace_size.argtypes = [c_int, c_int]
     L.snapkv_pool_topk.restype = c_int
@@ -251,6 +254,21 @@ def snapkv_compress_varlen(q_obs, k, v, seq_lens, pool_kernel: int, pool_type: i
         workspace.data_ptr(), workspace.numel(), _stream_ptr())
     _check(code, "snapkv_compress_varlen")
     return out_k, out_v, out_idx, workspace
+
+
+def snapkv_hit_counts(a_cur, idx, theta: float):
+    """a_cur fp32 [rows, n], idx int32 [rows, k] (CUDA) -> int32 [rows, 2]: per head the selected
+    positions above theta and all positions above theta (Eq. 3-7; H = ratio of the column sums)."""
+    if not (a_cur.is_cuda and a_cur.dtype == torch.float32 and a_cur.is_contiguous() and a_cur.dim() == 2):
+        raise SnapKVError("a_cur must be a contiguous CUDA fp32 [rows, n] tensor")
+    if not (idx.is_cuda and idx.dtype == torch.int32 and idx.is_contiguous() and idx.dim() == 2
+            and idx.shape[0] == a_cur.shape[0]):
+        raise SnapKVError("idx must be a contiguous CUDA int32 [rows, k] tensor")
+    out = torch.empty(a_cur.shape[0], 2, dtype=torch.int32, device=a_cur.device)
+    code = lib().snapkv_hit_counts(a_cur.data_ptr(), idx.data_ptr(), a_cur.shape[0], a_cur.shape[1],
+                                   idx.shape[1], float(theta), out.data_ptr(), _stream_ptr())
+    _check(code, "snapkv_hit_counts")
+    return out
 
 
 def snapkv_window_scores_lse(q_obs, k, lse_obs, out_vote=None, workspace=None):

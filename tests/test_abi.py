@@ -162,6 +162,13 @@ def test_varlen_entry_point_checks_every_sequence_before_launching(L):
     assert call(i32(1024, 600, 500), None, (FAKE, 1024)) == 3
 
 
+def test_hit_counts_rejects_bad_arguments(L):
+    assert L.snapkv_hit_counts(None, FAKE, 4, 100, 10, 0.5, FAKE, None) == 1
+    assert L.snapkv_hit_counts(FAKE, FAKE, 4, 100, 101, 0.5, FAKE, None) == 1   # k > n
+    assert L.snapkv_hit_counts(FAKE, FAKE, 0, 100, 10, 0.5, FAKE, None) == 1
+    assert L.snapkv_hit_counts(FAKE, FAKE, 70000, 100, 10, 0.5, FAKE, None) == 2
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(sk, "_lib", None)
     monkeypatch.setattr(sk, "LIB_PATH", "/nonexistent/libsnapkv.so")
