@@ -36,7 +36,8 @@ A second one, for grouped-query attention: group_votes / compress_grouped let th
 heads of a group select TOGETHER on the KV head they share (Eq. 1's sum runs over the
 window rows of all the group's heads), which keeps the compressed cache at Hkv heads.
 
-hit_counts / hit_rate state the paper's hit-rate measure of a selection (Sec. 3, Eq. 3-7).
+hit_counts / hit_rate state the paper's hit-rate measure of a selection (Sec. 3, Eq. 3-7);
+decode_attention is the generation step's attention over the compressed cache (Sec. 5.1.2).
 
 Every function here is pinned by tests that do not go through this file's own
 formulas (closed forms, invariants, library routines, brute force): see
@@ -372,3 +373,38 @@ def hit_rate(a_cur: np.ndarray, idx: np.ndarray, theta) -> float:
     """Eq. 7: H = sum(O) / sum(M_threshold_cur) over all heads (nan when nothing is important)."""
     c = hit_counts(a_cur, idx, theta)
     return float(c[:, 0].sum()) / float(c[:, 1].sum()) if c[:, 1].sum() > 0 else float("nan")
+
+
+def decode_attention(q_cur: np.ndarray, cache_k: np.ndarray, cache_v: np.ndarray):
+    """One generation step's attention over the compressed cache (Sec. 4.1: the compressed
+    keys and values are what later steps attend to; Sec. 5.1.2 measures exactly this
+    decoding).  bf16 bit patterns in: q_cur [B, Hq, d] (the generated token's queries),
+    cache_k / cache_v [B, Hc, R, d] with Hc dividing Hq (query head h reads cache head
+    h // (Hq // Hc): Hc = Hq for the expanded cache, Hc = Hkv for one selection per KV head).
+    Every cache row is visible (they all precede the generated token).  Returns fp64
+      out   [B, Hq, d]  sum_j p_j v_j,  p = softmax_j(q . k_j / sqrt(d))
+      lse   [B, Hq]     natural-log sum-exp of the logits
+      scale [B, Hq, d]  sum_j p_j |v_j|: the magnitude rounding errors are judged against.
+    """
+    B, Hq, d = q_cur.shape
+    _, Hc, R, _ = cache_k.shape
+    if Hq % Hc != 0 or cache_v.shape != cache_k.shape or cache_k.shape[0] != B or cache_k.shape[3] != d:
+        raise ValueError("shapes do not fit")
+    g = Hq // Hc
+    out = np.zeros((B, Hq, d), dtype=np.float64)
+    lse = np.zeros((B, Hq), dtype=np.float64)
+    scale = np.zeros((B, Hq, d), dtype=np.float64)
+    for b in range(B):
+        for h in range(Hq):
+            q = bf16_bits_to_f64(q_cur[b, h])
+            kf = bf16_bits_to_f64(cache_k[b, h // g])
+            vf = bf16_bits_to_f64(cache_v[b, h // g])
+            s = kf @ q / math.sqrt(d)
+            m = s.max()
+            e = np.exp(s - m)
+            z = e.sum()
+            p = e / z
+            out[b, h] = p @ vf
+            scale[b, h] = p @ np.abs(vf)
+            lse[b, h] = m + math.log(z)
+    return out, lse, scale
