@@ -289,6 +289,28 @@ snapkv_status_t snapkv_hit_counts(const float* a_cur, const int32_t* idx, int ro
                                   float theta, int32_t* out_counts, void* stream);
 
 /*
+ * One generation step's attention over the compressed cache (Sec. 5.1.2: decoding on the
+ * compressed keys and values; Sec. 4.1: later steps attend to what the step kept).
+ *   q_cur     bf16 [B, Hq, d]        device  the generated token's queries (post-RoPE)
+ *   cache_k/v bf16 [B, Hc, rows, d]  device  the compressed cache, every row visible; Hc
+ *             divides Hq and query head h reads cache head h / (Hq / Hc): Hc = Hq for the
+ *             output of snapkv_compress, Hc = Hkv for that of snapkv_compress_grouped
+ *   out       fp32 [B, Hq, d]        device  softmax_j(q . k_j / sqrt(d)) applied to the values
+ *   out_lse   fp32 [B, Hq] device or NULL: natural-log sum-exp of the logits (lets the
+ *             caller merge with attention over rows kept elsewhere, e.g. newly generated ones)
+ * bf16 products accumulated in fp32; the rows are split over many blocks and merged in a
+ * fixed order, so results are reproducible run to run.  `workspace`: device scratch of
+ * snapkv_decode_workspace_size(B, Hq, rows, d) bytes, 256-byte aligned (0 from the size
+ * query means unacceptable arguments).  Enqueued on `stream`: two kernels, no allocation.
+ * d must be 64 or 128 (SNAPKV_ERR_UNSUPPORTED otherwise), B * Hq <= 65535.
+ */
+size_t snapkv_decode_workspace_size(int B, int Hq, int rows, int d);
+snapkv_status_t snapkv_decode_attention(const void* q_cur, const void* cache_k, const void* cache_v,
+                                        int B, int Hq, int Hc, int rows, int d,
+                                        float* out, float* out_lse,
+                                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Synchronises `stream`, reads the status word the kernels keep at the start of
  * `workspace` and returns it (SNAPKV_OK or SNAPKV_ERR_TIMEOUT), or SNAPKV_ERR_CUDA
  * if the stream reports an error.  `detail`, if not NULL, receives a code telling

@@ -27,7 +27,7 @@ SYMBOLS = [
     "snapkv_last_launch_count", "snapkv_pool_topk_static",
     "snapkv_window_scores_lse", "snapkv_compress_lse", "snapkv_compress_strided",
     "snapkv_compress_grouped", "snapkv_compress_varlen",
-    "snapkv_hit_counts",
+    "snapkv_hit_counts", "snapkv_decode_workspace_size", "snapkv_decode_attention",
 ]
 
 _lib = None
@@ -73,6 +73,10 @@ def lib() -> ctypes.CDLL:
                                          + [c_vp, c_sz, c_vp])
     L.snapkv_hit_counts.restype = c_int
     L.snapkv_hit_counts.argtypes = [c_vp, c_vp, c_int, c_int, c_int, ctypes.c_float, c_vp, c_vp]
+    L.snapkv_decode_workspace_size.restype = c_sz
+    L.snapkv_decode_workspace_size.argtypes = [c_int] * 4
+    L.snapkv_decode_attention.restype = c_int
+    L.snapkv_decode_attention.argtypes = [c_vp] * 3 + [c_int] * 5 + [c_vp, c_vp, c_vp, c_sz, c_vp]
     L.snapkv_pool_topk_workspace_size.restype = c_sz
     L.snapkv_pool_topk_workspace_size.argtypes = [c_int, c_int]
     L.snapkv_pool_topk.restype = c_int
@@ -269,6 +273,27 @@ def snapkv_hit_counts(a_cur, idx, theta: float):
                                    idx.shape[1], float(theta), out.data_ptr(), _stream_ptr())
     _check(code, "snapkv_hit_counts")
     return out
+
+
+def snapkv_decode_attention(q_cur, cache_k, cache_v, workspace=None, want_lse: bool = True):
+    """q_cur bf16 [B, Hq, d], cache_k/v bf16 [B, Hc, rows, d] (CUDA, contiguous) ->
+    (out fp32 [B, Hq, d], lse fp32 [B, Hq] or None, workspace)."""
+    _dev_bf16(q_cur, "q_cur"), _dev_bf16(cache_k, "cache_k"), _dev_bf16(cache_v, "cache_v")
+    B, Hq, d = q_cur.shape
+    Bc, Hc, rows, dc = cache_k.shape
+    if Bc != B or dc != d or tuple(cache_v.shape) != tuple(cache_k.shape):
+        raise SnapKVError("q_cur, cache_k and cache_v disagree on their shapes")
+    L_ = lib()
+    need = L_.snapkv_decode_workspace_size(B, Hq, rows, d)
+    if workspace is None or workspace.numel() < need:
+        workspace = _alloc_ws(need, q_cur.device)
+    out = torch.empty(B, Hq, d, dtype=torch.float32, device=q_cur.device)
+    lse = torch.empty(B, Hq, dtype=torch.float32, device=q_cur.device) if want_lse else None
+    code = L_.snapkv_decode_attention(q_cur.data_ptr(), cache_k.data_ptr(), cache_v.data_ptr(), B, Hq, Hc,
+                                      rows, d, out.data_ptr(), lse.data_ptr() if want_lse else None,
+                                      workspace.data_ptr(), workspace.numel(), _stream_ptr())
+    _check(code, "snapkv_decode_attention")
+    return out, lse, workspace
 
 
 def snapkv_window_scores_lse(q_obs, k, lse_obs, out_vote=None, workspace=None):

@@ -169,6 +169,15 @@ def test_hit_counts_rejects_bad_arguments(L):
     assert L.snapkv_hit_counts(FAKE, FAKE, 70000, 100, 10, 0.5, FAKE, None) == 2
 
 
+def test_decode_attention_rejects_bad_arguments(L):
+    assert L.snapkv_decode_workspace_size(1, 4, 256, 96) == 0
+    assert L.snapkv_decode_workspace_size(4, 32, 4096, 128) >= 4 * 32 * 130 * 4
+    assert L.snapkv_decode_attention(FAKE, FAKE, FAKE, 1, 6, 4, 256, 128, FAKE, None, FAKE, 1 << 30, None) == 1
+    assert L.snapkv_decode_attention(FAKE, FAKE, FAKE, 1, 4, 4, 256, 96, FAKE, None, FAKE, 1 << 30, None) == 2
+    assert L.snapkv_decode_attention(FAKE, None, FAKE, 1, 4, 4, 256, 128, FAKE, None, FAKE, 1 << 30, None) == 1
+    assert L.snapkv_decode_attention(FAKE, FAKE, FAKE, 1, 4, 4, 256, 128, FAKE, None, None, 0, None) == 3
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(sk, "_lib", None)
     monkeypatch.setattr(sk, "LIB_PATH", "/nonexistent/libsnapkv.so")
