@@ -15,8 +15,24 @@
  *   - All tensors are dense, row-major, in the stated shape; "bf16" is the 16-bit
  *     brain-float bit pattern.  Device pointers must be 16-byte aligned and must
  *     not alias one another.
- *   - The caller owns every buffer.  The library allocates no device memory and
- *     keeps no per-call state; it only caches, per process, driver entry points.
+ *   - The caller owns every buffer the entry points read or write.  The library itself
+ *     holds, for the life of the process: one fixed 16 MiB device array on every GPU
+ *     that loads it (the scratch of snapkv_pool_topk_static), and, per device and
+ *     created on the first snapkv_compress_host call there, one side stream and a
+ *     handful of events.  It caches driver entry points, the SM count and "attribute
+ *     set" flags per device.  Nothing else is allocated and no per-call state is kept.
+ *   - One call at a time per device.  The scoring kernel behind snapkv_compress*,
+ *     snapkv_window_scores* is a persistent grid of one block per SM whose blocks wait
+ *     for one another's partial results; that is safe because all of them are resident
+ *     at once, which needs the whole GPU.  If another kernel holds SMs (a second
+ *     library call on another stream, other work of the caller, another tenant of the
+ *     GPU), blocks of the grid may not get an SM while the resident ones wait for them:
+ *     the waits then run into their one-second limit, the call's outputs are left
+ *     unwritten and SNAPKV_ERR_TIMEOUT is recorded in the status block.  So do not let
+ *     two scoring/compress calls, or such a call and other large kernels, overlap on one
+ *     GPU; calls on one stream never do.  snapkv_compress_host in addition shares its
+ *     side stream and events among all calls on a device: one caller per device at a
+ *     time.
  *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
  *     default stream).  Calls return without synchronising unless stated.
  *   - Errors come back as a snapkv_status_t; nothing aborts or throws.  Argument

@@ -332,6 +332,9 @@ def snapkv_pool_topk(vote, pool_kernel: int, pool_type: int, ksel: int, out_idx=
     L_ = lib()
     if out_idx is None:
         out_idx = torch.empty(rows, max(ksel, 0), dtype=torch.int32, device=vote.device)
+    elif not (out_idx.is_cuda and out_idx.dtype == torch.int32 and out_idx.is_contiguous()
+              and tuple(out_idx.shape) == (rows, ksel)):
+        raise SnapKVError("out_idx must be a contiguous CUDA int32 [rows, ksel] tensor")
     need = L_.snapkv_pool_topk_workspace_size(rows, n)
     if need and (workspace is None or workspace.numel() < need):
         workspace = _alloc_ws(need, vote.device)
@@ -352,6 +355,10 @@ def snapkv_pool_topk_static(vote, pool_kernel: int, pool_type: int, ksel: int, o
     if not (vote.is_cuda and vote.dtype == torch.float32 and vote.is_contiguous() and vote.dim() == 2):
         raise SnapKVError("vote must be a contiguous CUDA fp32 [rows, n] tensor")
     rows, n = vote.shape
+    if not (torch.is_tensor(out_idx) and out_idx.is_cuda and out_idx.dtype == torch.int32
+            and out_idx.is_contiguous() and tuple(out_idx.shape) == (rows, ksel)
+            and out_idx.device == vote.device):
+        raise SnapKVError("out_idx must be a contiguous CUDA int32 [rows, ksel] tensor on vote's device")
     code = lib().snapkv_pool_topk_static(vote.data_ptr(), rows, n, pool_kernel, pool_type, ksel,
                                          out_idx.data_ptr(), _stream_ptr())
     _check(code, "snapkv_pool_topk_static")

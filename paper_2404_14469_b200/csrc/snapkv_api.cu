@@ -33,6 +33,17 @@ static cudaError_t launch_clear(uint8_t* ws, const WorkspaceLayout& w, cudaStrea
                     reinterpret_cast<uint4*>(ws + from), n16);
 }
 
+// Zeroes the status block alone.  Entry points that run several single-sequence steps on one
+// workspace do this once, up front, and then run every step with keep_status set, so that the
+// block ends up holding the first error of any step.
+static cudaError_t clear_status(void* ws, cudaStream_t s) {
+  return cudaMemsetAsync(ws, 0, STATUS_BYTES, s);
+}
+
+static bool workspace_ok(const void* ws, size_t bytes, size_t need) {
+  return ws && (reinterpret_cast<uintptr_t>(ws) & 255) == 0 && bytes >= need;
+}
+
 WorkspaceLayout make_layout(const ScorePlan& p, int B, int Hq, int n, bool need_vote,
                             bool need_pooled) {
   WorkspaceLayout w;
@@ -158,8 +169,7 @@ static snapkv_status_t window_scores_impl(const void* q_obs, const void* k, cons
   ScorePlan p;
   if (!make_score_plan(B, Hq, Hkv, L, d, W, &p)) return SNAPKV_ERR_UNSUPPORTED;
   const WorkspaceLayout w = make_layout(p, B, Hq, L - W, false, false);
-  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < w.total)
-    return SNAPKV_ERR_WORKSPACE;
+  if (!workspace_ok(workspace, workspace_bytes, w.total)) return SNAPKV_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // with a supplied normaliser the conversion kernel clears what the clear kernel would
@@ -258,6 +268,11 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
     if (launch_gather(k, v, ks, vs, nullptr, B, Ho, Hkv, L, d, W, n, budget, out_k, out_v, s,
                       &launches) != cudaSuccess)
       return SNAPKV_ERR_CUDA;
+    // no kernel of this path can time out, but a caller that passes a workspace may read its
+    // status afterwards: it must not find what an earlier use of the memory left there
+    if (!keep_status && workspace_ok(workspace, workspace_bytes, STATUS_BYTES) &&
+        clear_status(workspace, s) != cudaSuccess)
+      return SNAPKV_ERR_CUDA;
     g_last_launches = launches;
     return SNAPKV_OK;
   }
@@ -265,8 +280,7 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
   if (!make_score_plan(B, Hq, Hkv, L, d, W, &p)) return SNAPKV_ERR_UNSUPPORTED;
   const bool scratch = select_needs_scratch(n);
   const WorkspaceLayout w = make_layout(p, B, Hq, n, true, scratch);
-  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < w.total)
-    return SNAPKV_ERR_WORKSPACE;
+  if (!workspace_ok(workspace, workspace_bytes, w.total)) return SNAPKV_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   if (!lse_obs) {
     if (launch_clear(ws, w, s, keep_status) != cudaSuccess) return SNAPKV_ERR_CUDA;
@@ -278,8 +292,8 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
                            reinterpret_cast<int*>(ws + w.off_status),
                            reinterpret_cast<int*>(ws + w.off_counters),
                            reinterpret_cast<float*>(ws + w.off_partials),
-                           reinterpret_cast<float*>(ws + w.off_lse), s, &launches, lse_obs) !=
-      cudaSuccess)
+                           reinterpret_cast<float*>(ws + w.off_lse), s, &launches, lse_obs,
+                           keep_status) != cudaSuccess)
     return SNAPKV_ERR_CUDA;
   if (launch_pool_topk(vote, B * Ho, n, pool_kernel, pool_type, ksel, out_idx,
                        scratch ? reinterpret_cast<float*>(ws + w.off_pooled) : nullptr, s,
@@ -369,19 +383,28 @@ snapkv_status_t snapkv_compress_varlen(const void* q_obs, const void* k, const v
   if ((k_strides && !strides_ok(k_strides, d, &ks)) || (v_strides && !strides_ok(v_strides, d, &vs)))
     return SNAPKV_ERR_INVALID_ARG;
   if (lse_obs && (reinterpret_cast<uintptr_t>(lse_obs) & 3)) return SNAPKV_ERR_INVALID_ARG;
-  // every sequence is checked before the first launch
+  // every sequence, every pointer and the workspace are checked before the first launch
+  st = check_pool(pool_kernel, pool_type);
+  if (st != SNAPKV_OK) return st;
+  if (!aligned16(q_obs) || !aligned16(k) || !aligned16(v) || !aligned16(out_k) || !aligned16(out_v))
+    return SNAPKV_ERR_INVALID_ARG;
   for (int b = 0; b < B; ++b) {
     if (seq_lens[b] < W || seq_lens[b] > Lmax) return SNAPKV_ERR_INVALID_ARG;
     if (k_seq_offsets && (k_seq_offsets[b] < 0 || (k_seq_offsets[b] & 7))) return SNAPKV_ERR_INVALID_ARG;
     if (v_seq_offsets && (v_seq_offsets[b] < 0 || (v_seq_offsets[b] & 7))) return SNAPKV_ERR_INVALID_ARG;
+    if (!out_idx && seq_lens[b] > W) return SNAPKV_ERR_INVALID_ARG;
   }
   for (int b = 0; b < B; ++b) {
     if (budget >= seq_lens[b]) continue;  // copied through: no scratch
     const size_t need =
         snapkv_workspace_size(1, Hq, Hkv, seq_lens[b], d, W, pool_kernel, pool_type, budget);
     if (need == 0) return SNAPKV_ERR_INVALID_ARG;
-    if (!workspace || workspace_bytes < need) return SNAPKV_ERR_WORKSPACE;
+    if (!workspace_ok(workspace, workspace_bytes, need)) return SNAPKV_ERR_WORKSPACE;
   }
+  // one clear of the status block for the whole call, whichever path the first sequence takes
+  const bool have_ws = workspace_ok(workspace, workspace_bytes, STATUS_BYTES);
+  if (have_ws && clear_status(workspace, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return SNAPKV_ERR_CUDA;
   const size_t head_rows = static_cast<size_t>(Hq) * budget * d * 2;  // bytes of one sequence's out_k
   int launches = 0;
   for (int b = 0; b < B; ++b) {
@@ -396,7 +419,7 @@ snapkv_status_t snapkv_compress_varlen(const void* q_obs, const void* k, const v
                        static_cast<uint8_t*>(out_k) + b * head_rows,
                        static_cast<uint8_t*>(out_v) + b * head_rows,
                        out_idx ? out_idx + static_cast<size_t>(b) * Hq * (budget - W) : nullptr,
-                       workspace, workspace_bytes, stream, b > 0,
+                       workspace, workspace_bytes, stream, /*keep_status=*/true,
                        lse_obs ? lse_obs + static_cast<size_t>(b) * Hq * W : nullptr, &ks, &vs);
     if (st != SNAPKV_OK) return st;
     launches += g_last_launches;
@@ -472,6 +495,9 @@ snapkv_status_t snapkv_compress_host(const void* q_obs, const void* k, const voi
   const size_t o_pair = static_cast<size_t>(g) * budget * d * 2;
   const size_t i_pair = static_cast<size_t>(g) * (budget - W) * 4;
   int launches = 0;
+  // (no workspace part in the staging buffer when the cache is copied through, budget >= L)
+  if (workspace_ok(dws, ws_bytes, STATUS_BYTES) && clear_status(dws, s) != cudaSuccess)
+    return SNAPKV_ERR_CUDA;
   for (int c = 0; c < parts; ++c) {
     const int p0 = c * per, np = (pairs - p0 < per) ? pairs - p0 : per;
     const size_t qo = p0 * q_pair, ko = p0 * k_pair, oo = p0 * o_pair, io = p0 * i_pair;
@@ -486,7 +512,8 @@ snapkv_status_t snapkv_compress_host(const void* q_obs, const void* k, const voi
     // over batch and KV head); the parts share the workspace, which the stream serialises
     const snapkv_status_t st = compress_impl(
         dq + qo, dk + ko, dv + ko, 1, np * g, np, L, d, W, pool_kernel, pool_type, budget,
-        dok + oo, dov + oo, reinterpret_cast<int32_t*>(di + io), dws, ws_bytes, stream, c > 0);
+        dok + oo, dov + oo, reinterpret_cast<int32_t*>(di + io), dws, ws_bytes, stream,
+        /*keep_status=*/true);
     if (st != SNAPKV_OK) return st;
     launches += g_last_launches;
     cudaStream_t back = s;

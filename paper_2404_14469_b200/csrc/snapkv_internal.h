@@ -4,6 +4,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <atomic>
+
 namespace snapkv {
 
 constexpr int TILE_KEYS = 128;      // keys per MMA tile
@@ -56,6 +58,30 @@ inline KVStrides dense_strides(int Hkv, int L, int d) {
   return KVStrides{static_cast<long long>(Hkv) * L * d, static_cast<long long>(L) * d, d};
 }
 
+// "Done once on this device" flag for set-up that belongs to a device's context (function
+// attributes).  done() and set() refer to the calling thread's current device; devices beyond
+// the table are never marked, so their set-up is simply repeated on every call.
+class DeviceOnce {
+ public:
+  bool done() const {
+    const int dev = current();
+    return dev >= 0 && flags_[dev].load(std::memory_order_acquire);
+  }
+  void set() {
+    const int dev = current();
+    if (dev >= 0) flags_[dev].store(true, std::memory_order_release);
+  }
+
+ private:
+  static constexpr int MAX_DEV = 64;
+  static int current() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEV) return -1;
+    return dev;
+  }
+  std::atomic<bool> flags_[MAX_DEV] = {};
+};
+
 struct WorkspaceLayout {
   size_t off_status, off_counters, off_partials, off_lse, off_vote, off_pooled, total;
 };
@@ -69,12 +95,14 @@ size_t select_scratch_bytes(int rows, int n);  // 0 when the rows fit one CTA
 // Enqueue both scoring passes.  `vote` is fp32 [B*Hq, n].  `counters` must be zero when the
 // kernel starts (the callers clear it together with the status block).  With `lse_obs`
 // (device fp32 [B*Hq, W], natural-log sum-exp of every window row) the statistics pass is
-// skipped: a small kernel converts the rows first, then only the vote pass runs.
+// skipped: a small kernel converts the rows first, then only the vote pass runs; that kernel
+// also zeroes the status block unless `keep_status` is set.
 cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrides& ks, int B,
                                  int Hq, int Hkv, int L, int d, int W, const ScorePlan& plan,
                                  float* vote, int* status,
                                  int* counters, float* partials, float* lse2, cudaStream_t stream,
-                                 int* launches, const float* lse_obs = nullptr);
+                                 int* launches, const float* lse_obs = nullptr,
+                                 bool keep_status = false);
 
 // Pool + top-k over `rows` rows of fp32 votes.  `pooled_scratch` (select_scratch_bytes bytes)
 // is only touched when select_needs_scratch(n).  With gsum > 1 a selection row is the sum of

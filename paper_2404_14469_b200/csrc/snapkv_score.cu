@@ -768,13 +768,15 @@ int sm_count() {
 // and marks every unit as merged, so the scoring kernel runs its vote phases only.
 constexpr int COUNTER_READY = 1 << 30;
 __global__ void lse_prep_kernel(const float* __restrict__ lse_obs, float* __restrict__ lse2,
-                                int* __restrict__ counters, int* __restrict__ status, int units,
-                                int sub_per_kv, int g, int hpu, int W, int ncols) {
+                                int* __restrict__ counters, int* __restrict__ status,
+                                int keep_status, int units, int sub_per_kv, int g, int hpu, int W,
+                                int ncols) {
   pdl_launch_dependents();
   pdl_wait();
   const int u = blockIdx.x, c = threadIdx.x;  // one block per unit, one thread per column
-  // this kernel stands in for the clear kernel of the two-sweep path: the status block too
-  if (u == 0 && c < STATUS_BYTES / 4) status[c] = 0;
+  // this kernel stands in for the clear kernel of the two-sweep path: the status block too,
+  // unless an earlier part of the same logical call may have left an error there
+  if (u == 0 && c < STATUS_BYTES / 4 && !keep_status) status[c] = 0;
   if (u >= units || c >= MAX_COLS) return;
   const int ukv = u / sub_per_kv;
   const int hq0 = ukv * g + (u - ukv * sub_per_kv) * hpu;  // flat over the batch
@@ -790,13 +792,13 @@ __global__ void lse_prep_kernel(const float* __restrict__ lse_obs, float* __rest
 template <int D, int NCH, bool SPLIT>
 cudaError_t run_scores(const CUtensorMap& tmK, const CUtensorMap& tmQ, const ScoreArgs& a,
                        int grid, cudaStream_t stream, int* launches) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static DeviceOnce once;  // one flag set per instantiation: the attribute is per function and device
+  if (!once.done()) {
     cudaError_t e = cudaFuncSetAttribute(score_kernel<D, NCH, SPLIT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          Smem<D>::DYN_BYTES);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    once.set();
   }
   // One CTA per SM (the shared-memory footprint allows no second one), grid no larger
   // than the SM count: every CTA becomes resident as soon as the stream's earlier work
@@ -867,7 +869,7 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrid
                                  int Hq, int Hkv, int L, int d, int W, const ScorePlan& plan,
                                  float* vote, int* status,
                                  int* counters, float* partials, float* lse2, cudaStream_t stream,
-                                 int* launches, const float* lse_obs) {
+                                 int* launches, const float* lse_obs, bool keep_status) {
   CUtensorMap tmK, tmQ;
   {
     // (d, position, KV head, batch) with the caller's strides: any layout whose rows of d
@@ -916,7 +918,8 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrid
   if (lse_obs) {
     const cudaError_t e =
         launch_pdl(lse_prep_kernel, dim3(plan.units), dim3(MAX_COLS), 0, stream, lse_obs, lse2,
-                   counters, status, plan.units, plan.sub_per_kv, plan.g, plan.hpu, W, plan.ncols);
+                   counters, status, keep_status ? 1 : 0, plan.units, plan.sub_per_kv, plan.g,
+                   plan.hpu, W, plan.ncols);
     if (e != cudaSuccess) return e;
     *launches += 1;
   }

@@ -31,24 +31,26 @@ __device__ __forceinline__ uint32_t float_to_key(float x) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-// Exclusive prefix sum of one int per thread over the block; returns the prefix and
-// leaves the block total in *total_s after the second barrier.
-__device__ __forceinline__ int block_exclusive_scan(int x, int* warp_sums_s, int* total_s) {
+// Exclusive prefix sum of one value per thread over the block (SEL_WARPS warps); returns the
+// prefix and leaves the block total in *total_s after the second barrier.  T is int, or
+// uint32_t when two 16-bit counts travel in one word: unsigned sums wrap, they never overflow.
+template <typename T>
+__device__ __forceinline__ T block_exclusive_scan(T x, T* warp_sums_s, T* total_s) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int inc = x;
+  T inc = x;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    const int y = __shfl_up_sync(0xffffffffu, inc, o);
+    const T y = __shfl_up_sync(0xffffffffu, inc, o);
     if (lane >= o) inc += y;
   }
   if (lane == 31) warp_sums_s[warp] = inc;
   __syncthreads();
   if (warp == 0) {
-    int w = warp_sums_s[lane];
-    int winc = w;
+    T w = warp_sums_s[lane];
+    T winc = w;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int y = __shfl_up_sync(0xffffffffu, winc, o);
+      const T y = __shfl_up_sync(0xffffffffu, winc, o);
       if (lane >= o) winc += y;
     }
     warp_sums_s[lane] = winc - w;  // exclusive
@@ -453,9 +455,17 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int gsum, int r, in
     cg += __popc(m_gt[wd]);
     ce += __popc(m_eq[wd]);
   }
-  const int packed = block_exclusive_scan((cg << 16) | ce, warp_sums, &scan_total);
-  int eq_before = packed & 0xffff;
-  int out_pos = (packed >> 16) + min(eq_before, need_eq);
+  // Two counts in one scan: keys above the threshold in the high half, keys equal to it in
+  // the low half.  Either total is at most n <= FAST_MAX_KEYS < 65536, so the low half never
+  // carries into the high one, and the word is unsigned so that a high half of 32768 or more
+  // (ksel that large is valid) stays a count after the shift.
+  static_assert(FAST_MAX_KEYS < 65536, "two 16-bit counts share one scan word");
+  uint32_t* scan_u = reinterpret_cast<uint32_t*>(warp_sums);
+  const uint32_t packed =
+      block_exclusive_scan<uint32_t>((static_cast<uint32_t>(cg) << 16) | static_cast<uint32_t>(ce),
+                                     scan_u, reinterpret_cast<uint32_t*>(&scan_total));
+  int eq_before = static_cast<int>(packed & 0xffffu);
+  int out_pos = static_cast<int>(packed >> 16) + min(eq_before, need_eq);
   int32_t* orow = out_idx + static_cast<size_t>(row) * ksel;
 #pragma unroll
   for (int wd = 0; wd < MASK_WORDS; ++wd) {
@@ -655,8 +665,7 @@ wide_count_kernel(int n, WideBufs wb) {
 // to it until ksel positions are out, in ascending position.
 __global__ void __launch_bounds__(WIDE_THREADS)
 wide_write_kernel(int n, int ksel, int32_t* __restrict__ out_idx, WideBufs wb) {
-  __shared__ int warp_sums[SEL_WARPS];
-  __shared__ int scan_total;
+  __shared__ int warp_sums[WIDE_THREADS / 32];
   const int row = blockIdx.y;
   const uint32_t T = static_cast<uint32_t>(wb.state[row * 8 + 0]);
   const int need_eq = wb.state[row * 8 + 2];
@@ -685,10 +694,12 @@ wide_write_kernel(int n, int ksel, int32_t* __restrict__ out_idx, WideBufs wb) {
     m_gt |= static_cast<uint32_t>(in && key > T) << i;
     m_eq |= static_cast<uint32_t>(in && key == T) << i;
   }
-  // block scan over 256 threads: block_exclusive_scan expects SEL_WARPS warp slots
+  // Block scan over the 8 warps of this kernel, two counts in one word: keys above the
+  // threshold in the high half, keys equal to it in the low half.  A chunk has WIDE_CHUNK =
+  // 8192 positions, so either half stays below 2^14 and the packed sums never carry or reach
+  // the sign bit; what came before the chunk is added outside the packed word.
+  static_assert(WIDE_CHUNK < 32768, "two counts of a chunk share one signed scan word");
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (threadIdx.x < SEL_WARPS) warp_sums[threadIdx.x] = 0;
-  __syncthreads();
   int x = (__popc(m_gt) << 16) | __popc(m_eq);
   int inc = x;
 #pragma unroll
@@ -701,7 +712,6 @@ wide_write_kernel(int n, int ksel, int32_t* __restrict__ out_idx, WideBufs wb) {
   int wpre = 0;
   for (int w2 = 0; w2 < warp; ++w2) wpre += warp_sums[w2];
   const int packed = wpre + inc - x;
-  (void)scan_total;
   int eq_seen = eq_before + (packed & 0xffff);
   int out_pos = gt_before + (packed >> 16) + min(eq_seen, need_eq);
   int32_t* orow = out_idx + static_cast<size_t>(row) * ksel;
@@ -726,6 +736,11 @@ __global__ void iota_kernel(int32_t* out, int rows, int n, int row_stride) {
 
 }  // namespace
 
+static DeviceOnce& select_attr_once() {
+  static DeviceOnce once;
+  return once;
+}
+
 static inline int key_slot4_host(int j) { return j + ((j >> 5) << 2); }
 constexpr int FAST_SMEM_BYTES = (FAST_MAX_KEYS + FAST_MAX_KEYS / 8 + 64) * 4;
 
@@ -744,8 +759,10 @@ size_t select_scratch_bytes(int rows, int n) {
 cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel, int pool_type,
                              int ksel, int32_t* out_idx, float* pooled_scratch,
                              cudaStream_t stream, int* launches, int gsum) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  // the opt-in to more than 48 KB of dynamic shared memory is a property of the device's
+  // context, so it is made once per device
+  DeviceOnce& once = select_attr_once();
+  if (!once.done()) {
     cudaError_t e = cudaFuncSetAttribute(pool_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          SEL_SMEM_KEYS * 4);
     if (e != cudaSuccess) return e;
@@ -757,7 +774,7 @@ cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel
     SNAPKV_FAST_ATTR(2, 0) SNAPKV_FAST_ATTR(2, 1) SNAPKV_FAST_ATTR(3, 0) SNAPKV_FAST_ATTR(3, 1)
     SNAPKV_FAST_ATTR(6, 0) SNAPKV_FAST_ATTR(6, 1)
 #undef SNAPKV_FAST_ATTR
-    attr_done = true;
+    once.set();
   }
   const int r = pool_kernel >> 1;
   if (n <= FAST_MAX_KEYS && r <= 7) {

@@ -83,3 +83,34 @@ def test_packed_cache_with_supplied_lse_matches_per_sequence_oracle():
         for b, s in enumerate(seqs):
             _check_sequence(b, s, lens[b], W, kernel, "max", budget, out_k, out_v, out_idx,
                             lse=lses[b].astype(np.float64) if use_lse else None)
+
+
+@pytest.mark.parametrize("use_lse", [False, True])
+def test_status_block_is_clean_whichever_path_the_first_sequence_takes(use_lse):
+    # first sequence shorter than the budget (copied through), second one compressed; the
+    # workspace arrives full of 0xFF, as memory that was never cleared may
+    lens, Hq, Hkv, d, W, kernel, budget = [129, 1000], 4, 2, 128, 32, 5, 200
+    seqs = _sequences(lens, Hq, Hkv, d, W, kernel, "avg", budget, seed=3)
+    B, Lmax = len(lens), max(lens)
+    k = torch.zeros(B, Hkv, Lmax, d, dtype=torch.bfloat16)
+    v = torch.zeros(B, Hkv, Lmax, d, dtype=torch.bfloat16)
+    for b, s in enumerate(seqs):
+        k[b, :, :lens[b]] = s["k"][0]
+        v[b, :, :lens[b]] = s["v"][0]
+    q = torch.cat([s["q_obs"] for s in seqs])
+    lses = [orc.lse_obs(_bits(s["q_obs"]), _bits(s["k"])).astype(np.float32) for s in seqs]
+    lse = torch.from_numpy(np.concatenate(lses)).cuda() if use_lse else None
+    need = sk.snapkv_workspace_size(1, Hq, Hkv, Lmax, d, W, kernel, sk.POOL_AVG, budget)
+    ws = torch.full((need,), 0xFF, dtype=torch.uint8, device="cuda")
+    out_k, out_v, out_idx, ws2 = sk.snapkv_compress_varlen(q.cuda(), k.cuda(), v.cuda(), lens, kernel,
+                                                           sk.POOL_AVG, budget, lse_obs=lse, workspace=ws)
+    assert ws2 is ws
+    assert sk.snapkv_device_status(ws) == (sk.OK, 0)
+    for b, s in enumerate(seqs):
+        _check_sequence(b, s, lens[b], W, kernel, "avg", budget, out_k, out_v, out_idx,
+                        lse=lses[b].astype(np.float64) if use_lse else None)
+    # the same for a plain call that only copies the cache through
+    ws.fill_(0xFF)
+    dev = {x: seqs[0][x].cuda() for x in ("q_obs", "k", "v")}
+    sk.snapkv_compress(dev["q_obs"], dev["k"], dev["v"], kernel, sk.POOL_AVG, budget, workspace=ws)
+    assert sk.snapkv_device_status(ws) == (sk.OK, 0)

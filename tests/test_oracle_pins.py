@@ -232,28 +232,35 @@ def test_topk_nesting_across_budgets():
 
 
 # ---------------------------------------------------------------- whole step
-def _listing_with_library_ops(q_bits, k_bits, v_bits, W, budget, kernel, pool_type):
-    """Second, independent statement of the step with framework routines (softmax,
-    pool1d, topk, gather, cat), in the order of the paper's Listing 1, fp64, MHA."""
-    tq = torch.from_numpy(orc.bf16_bits_to_f64(q_bits))
-    tk = torch.from_numpy(orc.bf16_bits_to_f64(k_bits))
+def _step_head_by_head(q_bits, k_bits, v_bits, W, budget, kernel, pool_type):
+    """Second, independent statement of the whole step (Sec. 4, Eq. 1-2), MHA, fp64, one head
+    at a time: each window row is an ordinary attention row over the keys it may see
+    (library log-sum-exp), Eq. 1 adds the rows, a sliding-window view does the pooling, a
+    sort of (value, position) pairs ranks the positions, and the kept rows are picked by
+    plain indexing."""
+    tq = orc.bf16_bits_to_f64(q_bits)
+    tk = orc.bf16_bits_to_f64(k_bits)
     B, H, L, d = tk.shape
-    n = L - W
-    logits = tq @ tk.transpose(-1, -2) / math.sqrt(d)
-    mask = torch.full((L, L), float("-inf"), dtype=torch.float64).triu(1)[n:, :]
-    attn = torch.softmax(logits + mask, dim=-1)
-    vote = attn[..., :n].sum(dim=-2)
-    if pool_type == orc.POOL_MAX:
-        pooled = F.max_pool1d(vote, kernel_size=kernel, padding=kernel // 2, stride=1)
-    else:
-        pooled = F.avg_pool1d(vote, kernel_size=kernel, padding=kernel // 2, stride=1)
-    idx = pooled.topk(budget - W, dim=-1).indices
-    kb = torch.from_numpy(k_bits.astype(np.int32))
-    vb = torch.from_numpy(v_bits.astype(np.int32))
-    gi = idx.unsqueeze(-1).expand(-1, -1, -1, d)
-    ck = torch.cat([kb[..., :n, :].gather(2, gi), kb[..., n:, :]], dim=2)
-    cv = torch.cat([vb[..., :n, :].gather(2, gi), vb[..., n:, :]], dim=2)
-    return vote.numpy(), pooled.numpy(), idx.numpy(), ck.numpy(), cv.numpy()
+    n, r, ksel = L - W, kernel // 2, budget - W
+    vote = np.zeros((B, H, n))
+    pooled = np.zeros((B, H, n))
+    idx = np.zeros((B, H, ksel), dtype=np.int64)
+    ck = np.zeros((B, H, budget, d), dtype=np.uint16)
+    cv = np.zeros((B, H, budget, d), dtype=np.uint16)
+    for b, h in itertools.product(range(B), range(H)):
+        for i in range(W):
+            seen = n + i + 1                                    # the prefix and the window up to row i
+            row = torch.from_numpy(tk[b, h, :seen] @ tq[b, h, i]) / math.sqrt(d)
+            vote[b, h] += torch.exp(row - torch.logsumexp(row, dim=0)).numpy()[:n]
+        padded = np.concatenate([np.zeros(r), vote[b, h], np.zeros(r)])   # votes are >= 0
+        windows = np.lib.stride_tricks.sliding_window_view(padded, kernel)
+        pooled[b, h] = windows.max(axis=1) if pool_type == orc.POOL_MAX else windows.sum(axis=1) / kernel
+        ranked = sorted(range(n), key=lambda j: pooled[b, h, j], reverse=True)
+        idx[b, h] = np.array(ranked[:ksel])
+        keep = np.sort(idx[b, h])
+        ck[b, h] = np.concatenate([k_bits[b, h, keep], k_bits[b, h, n:]])
+        cv[b, h] = np.concatenate([v_bits[b, h, keep], v_bits[b, h, n:]])
+    return vote, pooled, idx, ck, cv
 
 
 @pytest.mark.parametrize("pool_type,kernel", [(orc.POOL_MAX, 7), (orc.POOL_AVG, 5), (orc.POOL_MAX, 1)])
@@ -262,7 +269,7 @@ def test_whole_step_against_library_ops(pool_type, kernel):
     w = synth.make_random(2, 3, 3, 150, 32, W, seed=14, q_scale=2.0)
     q, k, v = (synth.bf16_bits(w[x]) for x in ("q_obs", "k", "v"))
     res = orc.compress(q, k, v, kernel, pool_type, budget)
-    vote, pooled, idx, ck, cv = _listing_with_library_ops(q, k, v, W, budget, kernel, pool_type)
+    vote, pooled, idx, ck, cv = _step_head_by_head(q, k, v, W, budget, kernel, pool_type)
     assert np.allclose(res["vote"], vote, rtol=1e-12)
     assert np.allclose(res["pooled"], pooled, rtol=1e-12)
     ksel = budget - W
