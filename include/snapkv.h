@@ -334,6 +334,50 @@ snapkv_status_t snapkv_decode_attention(const void* q_cur, const void* cache_k, 
  */
 snapkv_status_t snapkv_device_status(const void* workspace, void* stream, int* detail);
 
+/*
+ * The scoring kernel's schedule, for inspection (no counterpart in the paper).  The kernel
+ * is a persistent grid; every block walks a fixed list of work items - tiles [t0, t1) of 128
+ * keys of one unit (a batch, a KV head and up to 128 window columns of its query heads), in
+ * the statistics sweep or in the vote sweep of Eq. 1 - and the blocks that share a unit's
+ * statistics sweep each publish one partial (slot s of nseg).  This routine runs the
+ * kernel's own item walk on the host for block `cta` of `grid`: it writes up to max_items
+ * records of six int32 {unit, t0, t1, vote (0/1), slot, nseg} to out_items (host memory)
+ * and returns the number of items, or -1 if the arguments are not acceptable.  out_plan,
+ * if not NULL, receives eight int32: units, units per wave, waves, tiles per unit in the
+ * statistics sweep, tiles per unit in the vote sweep, partial slots per unit, waves the
+ * statistics run ahead of the votes, window columns per unit.  Host only, no CUDA calls.
+ */
+int snapkv_schedule_items(int B, int Hq, int Hkv, int L, int d, int W, int votes_only,
+                          int grid, int cta, int32_t* out_items, int max_items,
+                          int32_t* out_plan);
+
+/*
+ * Time limit of the device-side waits (no counterpart in the paper; the scoring kernel's
+ * blocks wait for one another's partial softmax statistics of Eq. 1's normaliser, and for
+ * their own copies and tensor-core operations).  Every such wait gives up after `limit_ns`
+ * nanoseconds (one second unless changed; values below one millisecond are raised to
+ * that); a wait on another block gives up after half of it, so that the detail word
+ * names the wait that failed and not one downstream of it.  Process-wide, applies to
+ * kernels launched afterwards, returns the previous limit.  Host only.
+ */
+unsigned long long snapkv_set_wait_limit_ns(unsigned long long limit_ns);
+
+/*
+ * Self-test of the time-out path (no counterpart in the paper).  Same arguments as
+ * snapkv_window_scores, but only the vote sweep is launched and nothing ever supplies the
+ * softmax statistics it waits for: every block's wait runs into the limit, the blocks drain
+ * their copies, release tensor memory and return; out_vote is left unwritten.  Afterwards
+ * snapkv_device_status(workspace) reports SNAPKV_ERR_TIMEOUT with detail 7 (the wait for a
+ * unit's statistics) and the context is usable as before.  The call occupies the GPU for
+ * about half the wait limit: lower the limit first (snapkv_set_wait_limit_ns) and restore
+ * it afterwards.
+ */
+snapkv_status_t snapkv_selftest_stalled_scores(const void* q_obs, const void* k,
+                                               int B, int Hq, int Hkv, int L, int d, int W,
+                                               float* out_vote,
+                                               void* workspace, size_t workspace_bytes,
+                                               void* stream);
+
 /* Number of kernel launches the last successful snapkv_compress /
  * snapkv_window_scores call of this thread enqueued (for accounting in benchmarks).
  * Host only. */

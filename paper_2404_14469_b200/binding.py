@@ -28,6 +28,7 @@ SYMBOLS = [
     "snapkv_window_scores_lse", "snapkv_compress_lse", "snapkv_compress_strided",
     "snapkv_compress_grouped", "snapkv_compress_varlen",
     "snapkv_hit_counts", "snapkv_decode_workspace_size", "snapkv_decode_attention",
+    "snapkv_set_wait_limit_ns", "snapkv_selftest_stalled_scores", "snapkv_schedule_items",
 ]
 
 _lib = None
@@ -93,6 +94,13 @@ def lib() -> ctypes.CDLL:
     L.snapkv_device_status.argtypes = [c_vp, c_vp, ctypes.POINTER(c_int)]
     L.snapkv_last_launch_count.restype = c_int
     L.snapkv_last_launch_count.argtypes = []
+    L.snapkv_schedule_items.restype = c_int
+    L.snapkv_schedule_items.argtypes = [c_int] * 9 + [ctypes.POINTER(ctypes.c_int32), c_int,
+                                                      ctypes.POINTER(ctypes.c_int32)]
+    L.snapkv_set_wait_limit_ns.restype = ctypes.c_ulonglong
+    L.snapkv_set_wait_limit_ns.argtypes = [ctypes.c_ulonglong]
+    L.snapkv_selftest_stalled_scores.restype = c_int
+    L.snapkv_selftest_stalled_scores.argtypes = L.snapkv_window_scores.argtypes
     _lib = L
     return L
 
@@ -320,6 +328,44 @@ def snapkv_window_scores(q_obs, k, out_vote=None, workspace=None, lse_obs=None):
         code = L_.snapkv_window_scores_lse(q_obs.data_ptr(), k.data_ptr(),
                                            _lse_arg(lse_obs, B, Hq, W), *tail)
     _check(code, "snapkv_window_scores")
+    return out_vote, workspace
+
+
+def snapkv_schedule_items(B, Hq, Hkv, L, d, W, grid, cta, votes_only=False):
+    """The scoring kernel's work items for block `cta` of `grid` (host only).  Returns
+    (items, plan): items is a list of (unit, t0, t1, vote, slot, nseg); plan a dict."""
+    L_ = lib()
+    plan = (ctypes.c_int32 * 8)()
+    n = L_.snapkv_schedule_items(B, Hq, Hkv, L, d, W, int(votes_only), grid, cta, None, 0, plan)
+    if n < 0:
+        raise SnapKVError("snapkv_schedule_items: arguments not acceptable")
+    buf = (ctypes.c_int32 * (6 * max(n, 1)))()
+    L_.snapkv_schedule_items(B, Hq, Hkv, L, d, W, int(votes_only), grid, cta, buf, n, plan)
+    items = [tuple(buf[6 * i:6 * i + 6]) for i in range(n)]
+    names = ("units", "units_per_wave", "waves", "tiles_stats", "tiles_vote", "maxseg", "lag", "ncols")
+    return items, dict(zip(names, plan))
+
+
+def snapkv_set_wait_limit_ns(limit_ns: int) -> int:
+    """Sets the time limit of device-side waits; returns the previous one."""
+    return int(lib().snapkv_set_wait_limit_ns(int(limit_ns)))
+
+
+def snapkv_selftest_stalled_scores(q_obs, k, out_vote=None, workspace=None):
+    """Launches the vote sweep with statistics that never arrive (time-out self-test).
+    Returns (out_vote, workspace); read the outcome with snapkv_device_status."""
+    _dev_bf16(q_obs, "q_obs"), _dev_bf16(k, "k")
+    B, Hq, Hkv, L, d, W = _shapes(q_obs, k)
+    L_ = lib()
+    if out_vote is None:
+        out_vote = torch.empty(B, Hq, L - W, dtype=torch.float32, device=k.device)
+    need = L_.snapkv_workspace_size(B, Hq, Hkv, L, d, W, 1, 0, W + 1)
+    if workspace is None or workspace.numel() < need:
+        workspace = _alloc_ws(need, k.device)
+    code = L_.snapkv_selftest_stalled_scores(q_obs.data_ptr(), k.data_ptr(), B, Hq, Hkv, L, d, W,
+                                             out_vote.data_ptr(), workspace.data_ptr(),
+                                             workspace.numel(), _stream_ptr())
+    _check(code, "snapkv_selftest_stalled_scores")
     return out_vote, workspace
 
 

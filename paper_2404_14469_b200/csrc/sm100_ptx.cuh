@@ -1,6 +1,6 @@
 // Thin inline-PTX wrappers for the sm_100a features the scoring kernels use:
 // mbarrier, TMA tiled loads (cp.async.bulk.tensor), tcgen05 MMA / TMEM.
-// Every wait here is bounded: it gives up after WAIT_LIMIT_NS and reports failure,
+// Every wait here is bounded: it gives up after the CTA's wait limit and reports failure,
 // so a kernel can stop, release its TMEM and return with an error status.
 #pragma once
 #include <cuda.h>
@@ -9,7 +9,14 @@
 
 namespace snapkv {
 
-constexpr unsigned long long WAIT_LIMIT_NS = 1000ull * 1000ull * 1000ull;  // 1 s
+constexpr unsigned long long DEFAULT_WAIT_LIMIT_NS = 1000ull * 1000ull * 1000ull;  // 1 s
+
+// A CTA keeps two words of wait control in shared memory: an abort flag (0 = running, else
+// the code of the wait that gave up first) and, 8 bytes behind it, the time limit of a wait in
+// nanoseconds.  The wait helpers take the flag's address and find the limit from it.
+__device__ __forceinline__ unsigned long long wait_limit_ns(volatile int* abort_flag) {
+  return *reinterpret_cast<volatile unsigned long long*>(abort_flag + 1);
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -61,7 +68,7 @@ __device__ __forceinline__ bool mbar_wait_thread(uint32_t bar, uint32_t parity,
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag != 0) return false;
-    if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+    if (globaltimer_ns() - t0 > wait_limit_ns(abort_flag)) {
       *abort_flag = code;
       return false;
     }
@@ -81,7 +88,7 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity,
     int stop = 0;
     if ((threadIdx.x & 31) == 0) {
       if (*abort_flag != 0) stop = 1;
-      else if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = code; stop = 1; }
+      else if (globaltimer_ns() - t0 > wait_limit_ns(abort_flag)) { *abort_flag = code; stop = 1; }
     }
     if (__shfl_sync(0xffffffffu, stop, 0)) return false;
   }
@@ -99,14 +106,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* m, 
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
       "[%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y)
-      : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* m, uint32_t bar,
-                                            int x, int y, int z) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
-      "[%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y), "r"(z)
       : "memory");
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* m, uint32_t bar,
@@ -131,14 +130,6 @@ __device__ __forceinline__ void fence_proxy_async() {
   asm volatile("fence.proxy.async;" ::: "memory");
 }
 // The same load with an L2 eviction policy (from l2_policy_evict_first).
-__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* m, uint32_t bar,
-                                                 int x, int y, int z, uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      ".L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y), "r"(z), "l"(policy)
-      : "memory");
-}
 __device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap* m, uint32_t bar,
                                                  int x, int y, int z, int w, uint64_t policy) {
   asm volatile(
@@ -191,7 +182,7 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, ui
 __device__ __forceinline__ void tmem_wait_ld() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
-// Each lane reads its own TMEM lane: 32 / 16 consecutive 32-bit columns.
+// Each lane reads its own TMEM lane: 32 consecutive 32-bit columns.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   uint32_t* r = reinterpret_cast<uint32_t*>(v);
   asm volatile(
@@ -206,18 +197,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
       : "r"(taddr)
       : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
-  uint32_t* r = reinterpret_cast<uint32_t*>(v);
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
-        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
-        "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-}
-
 // Shared-memory matrix descriptor for a K-major bf16 tile stored as rows of 128 bytes
 // with the 128-byte swizzle (the layout TMA writes with CU_TENSOR_MAP_SWIZZLE_128B):
 // groups of 8 rows are 1024 bytes apart.  `saddr` is the shared address of the tile
@@ -257,10 +236,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
-}
-
-__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
 }  // namespace snapkv

@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "../../include/snapkv.h"
@@ -66,6 +67,9 @@ WorkspaceLayout make_layout(const ScorePlan& p, int B, int Hq, int n, bool need_
 }
 
 static thread_local int g_last_launches = 0;
+
+static std::atomic<unsigned long long> g_wait_limit_ns{1000ull * 1000ull * 1000ull};
+unsigned long long wait_limit_setting() { return g_wait_limit_ns.load(std::memory_order_relaxed); }
 
 // Side stream and events of snapkv_compress_host, one set per device, created on first use
 // and kept for the life of the process (nullptr if they cannot be created: the entry point
@@ -536,6 +540,62 @@ snapkv_status_t snapkv_compress_host(const void* q_obs, const void* k, const voi
         cudaStreamWaitEvent(s, side->done, 0) != cudaSuccess)
       return SNAPKV_ERR_CUDA;
   }
+  g_last_launches = launches;
+  return SNAPKV_OK;
+}
+
+int snapkv_schedule_items(int B, int Hq, int Hkv, int L, int d, int W, int votes_only, int grid,
+                          int cta, int32_t* out_items, int max_items, int32_t* out_plan) {
+  if (check_common(B, Hq, Hkv, L, d, W) != SNAPKV_OK || W >= L) return -1;
+  if (grid < 1 || grid > MAX_GRID || cta < 0 || cta >= grid || max_items < 0) return -1;
+  if (max_items > 0 && !out_items) return -1;
+  ScorePlan p;
+  if (!make_score_plan(B, Hq, Hkv, L, d, W, &p)) return -1;
+  if (out_plan) {
+    out_plan[0] = p.units;
+    out_plan[1] = votes_only ? p.units : p.units_per_wave;
+    out_plan[2] = votes_only ? 1 : p.nwaves;
+    out_plan[3] = p.tiles_stats;
+    out_plan[4] = p.tiles_vote;
+    out_plan[5] = p.maxseg;
+    out_plan[6] = p.pipelined;
+    out_plan[7] = p.ncols;
+  }
+  return list_schedule_items(p, L, W, Hkv, votes_only ? 1 : 0, grid, cta, out_items, max_items);
+}
+
+unsigned long long snapkv_set_wait_limit_ns(unsigned long long limit_ns) {
+  // at least a millisecond: a limit near the length of an ordinary wait would turn a busy
+  // memory system into an error
+  if (limit_ns < 1000000ull) limit_ns = 1000000ull;
+  return g_wait_limit_ns.exchange(limit_ns, std::memory_order_relaxed);
+}
+
+snapkv_status_t snapkv_selftest_stalled_scores(const void* q_obs, const void* k, int B, int Hq,
+                                               int Hkv, int L, int d, int W, float* out_vote,
+                                               void* workspace, size_t workspace_bytes,
+                                               void* stream) {
+  snapkv_status_t st = check_common(B, Hq, Hkv, L, d, W);
+  if (st != SNAPKV_OK) return st;
+  if (W >= L || !q_obs || !k || !out_vote) return SNAPKV_ERR_INVALID_ARG;
+  if (!aligned16(q_obs) || !aligned16(k) || (reinterpret_cast<uintptr_t>(out_vote) & 3))
+    return SNAPKV_ERR_INVALID_ARG;
+  ScorePlan p;
+  if (!make_score_plan(B, Hq, Hkv, L, d, W, &p)) return SNAPKV_ERR_UNSUPPORTED;
+  const WorkspaceLayout w = make_layout(p, B, Hq, L - W, false, false);
+  if (!workspace_ok(workspace, workspace_bytes, w.total)) return SNAPKV_ERR_WORKSPACE;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int launches = 1;
+  // counters cleared and never raised: every unit looks as if its statistics were still
+  // on their way, for ever
+  if (launch_clear(ws, w, s) != cudaSuccess) return SNAPKV_ERR_CUDA;
+  cudaError_t e = launch_window_scores(
+      q_obs, k, dense_strides(Hkv, L, d), B, Hq, Hkv, L, d, W, p, out_vote,
+      reinterpret_cast<int*>(ws + w.off_status), reinterpret_cast<int*>(ws + w.off_counters),
+      reinterpret_cast<float*>(ws + w.off_partials), reinterpret_cast<float*>(ws + w.off_lse), s,
+      &launches, nullptr, false, /*never_ready=*/true);
+  if (e != cudaSuccess) return SNAPKV_ERR_CUDA;
   g_last_launches = launches;
   return SNAPKV_OK;
 }

@@ -22,7 +22,7 @@ enum WaitCode {
   WAIT_MMA_TMEM_EMPTY = 3,
   WAIT_EPI_TMEM_FULL = 4,
   WAIT_Q_FULL = 5,
-  WAIT_DRAIN = 6,
+  /* 6 is not used */
   WAIT_UNIT_STATS = 7,
   WAIT_PART_EMPTY = 8,
   WAIT_PART_FULL = 9,
@@ -86,6 +86,17 @@ struct WorkspaceLayout {
   size_t off_status, off_counters, off_partials, off_lse, off_vote, off_pooled, total;
 };
 
+// The work items of block `cta` of a grid of `grid` blocks, in the order the scoring kernel
+// walks them (the very routine the kernel runs, on the host).  Writes up to `max_items`
+// records {unit, first tile, end tile, 1 for the vote sweep, partial slot, partials of the unit}
+// and returns how many items there are.
+int list_schedule_items(const ScorePlan& plan, int L, int W, int Hkv, int votes_only, int grid,
+                        int cta, int32_t* out, int max_items);
+
+// Time limit, in nanoseconds, that kernels launched from now on give each of their device-side
+// waits (process-wide; one second unless snapkv_set_wait_limit_ns changed it).
+unsigned long long wait_limit_setting();
+
 bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* plan);
 WorkspaceLayout make_layout(const ScorePlan& p, int B, int Hq, int n, bool need_vote,
                             bool need_pooled);
@@ -96,13 +107,15 @@ size_t select_scratch_bytes(int rows, int n);  // 0 when the rows fit one CTA
 // kernel starts (the callers clear it together with the status block).  With `lse_obs`
 // (device fp32 [B*Hq, W], natural-log sum-exp of every window row) the statistics pass is
 // skipped: a small kernel converts the rows first, then only the vote pass runs; that kernel
-// also zeroes the status block unless `keep_status` is set.
+// also zeroes the status block unless `keep_status` is set.  `never_ready` (self-test of the
+// time-out path): the vote pass alone is launched and nothing marks the units' statistics as
+// present, so its wait for them must run out.
 cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrides& ks, int B,
                                  int Hq, int Hkv, int L, int d, int W, const ScorePlan& plan,
                                  float* vote, int* status,
                                  int* counters, float* partials, float* lse2, cudaStream_t stream,
                                  int* launches, const float* lse_obs = nullptr,
-                                 bool keep_status = false);
+                                 bool keep_status = false, bool never_ready = false);
 
 // Pool + top-k over `rows` rows of fp32 votes.  `pooled_scratch` (select_scratch_bytes bytes)
 // is only touched when select_needs_scratch(n).  With gsum > 1 a selection row is the sum of

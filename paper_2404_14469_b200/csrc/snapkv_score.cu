@@ -7,13 +7,13 @@
 //      (max, sum of exp) over the keys it sees: an online softmax without shuffles.
 //      When the unit has fewer than 128 window rows the rows are replicated along M and
 //      each replica takes a different slice of the tile's keys, so all four epilogue
-//      warps of a warpgroup stay busy.  Each CTA publishes one (max, sum) pair per window
-//      row for the keys it saw and bumps the unit's counter.
+//      warps of a warpgroup stay busy.  Each CTA publishes one log2-sum-exp per window row
+//      for the keys it saw (its "partial") and bumps the unit's counter.
 //  pass V (votes)       S tile = K_tile[128 x d] . Q[ncols x d]^T : keys on TMEM lanes,
 //      window rows on columns.  Once the unit's counter shows that every partial has been
-//      published, the CTA merges them into one log2-sum-exp per window row; then each
-//      thread owns one key and adds exp2(s*c - lse) over the W columns of each head: the
-//      sum over the window is a serial add per thread.
+//      published, the CTA folds them, in slot order, into one log2-sum-exp per window row;
+//      then each thread owns one key and adds exp2(s*c - lse) over the W columns of each
+//      head: the sum over the window is a serial add per thread.
 //
 // Units (batch, KV head, head sub-group) are grouped into waves small enough for L2; the
 // kernel walks the phases  S(0), S(1), V(0), S(2), V(1), ...  so that the second sweep
@@ -28,10 +28,9 @@
 // arithmetic; with 64 or more query columns per unit a second set of eight softmax warps
 // (12-19) takes every other tile, each warpgroup of a set working on half of the columns:
 // the epilogue is bound by instruction latency, and four warps per scheduler hide it where
-// two do not.  Warps 10 and 11 are the book-keepers: warp 10 merges and
-// publishes the partial statistics the softmax warps leave in shared memory, warp 11
-// fetches the merged log-sum-exp of the coming vote items while the softmax warps are
-// still busy.  The single-thread roles (TMA and MMA issue) are entered through elect.sync:
+// two do not.  Warps 10 and 11 are the book-keepers: warp 10 publishes the partial
+// statistics the softmax warps leave in shared memory, warp 11 fetches and folds the
+// partials of the coming vote items' units while the softmax warps are still busy.  The single-thread roles (TMA and MMA issue) are entered through elect.sync:
 // the compiler then keeps descriptors and addresses in uniform registers, which cut the
 // time per tcgen05.mma issue by about a third against a lane-index test.
 #include <cuda.h>
@@ -64,7 +63,7 @@ constexpr int threads_for(bool split) { return split ? 640 : 384; }
 constexpr long long WAVE_BYTES = static_cast<long long>(WAVE_MIB) << 20;
 constexpr int NPB = 2;                // buffers for partial statistics (book-keeper queue)
 constexpr int NLB = 8;                // buffers for merged log-sum-exp rows
-constexpr int MERGE_SEGS = 32;        // partials staged in shared memory per merge round
+constexpr int MERGE_SEGS = 40;        // partials staged in shared memory per merge round
 
 struct ScoreArgs {
   int L, n, W, Hkv;
@@ -75,10 +74,11 @@ struct ScoreArgs {
   int maxseg;               // partial slots per unit
   int pipelined;            // how many waves the statistics run ahead of the votes (>= 1)
   int votes_only;           // 1: lse2 and the counters are already set, no statistics pass
+  unsigned long long wait_ns;  // time limit of every device-side wait
   float c2;                 // log2(e) / sqrt(d)
   float* partials;          // [units][maxseg][MAX_COLS] log2-sum-exp of one CTA's share
-  float* lse2;              // [units][MAX_COLS] minus the merged log2-sum-exp per window row
-  int* counters;            // [units] published partials (+1 once lse2 is written)
+  float* lse2;              // [units][MAX_COLS] minus the log2-sum-exp per window row, when supplied
+  int* counters;            // [units] published partials (a large value when lse2 was supplied)
   int* status;
   float* vote;
 };
@@ -95,7 +95,7 @@ struct Smem {
   // pfull[NPB], pempty[NPB] (partial statistics), lfull[NLB], lempty[NLB] (log-sum-exp),
   // merge (bulk copy of a unit's partials)
   static constexpr int NBAR = 2 * STAGES + 2 * NBUF + 5 + 2 * NPB + 2 * NLB + 1;
-  static constexpr int OFF_MISC = OFF_BAR + ((NBAR * 8 + 15) & ~15);  // tmem ptr, abort
+  static constexpr int OFF_MISC = OFF_BAR + ((NBAR * 8 + 15) & ~15);  // tmem ptr, abort flag, wait limit
   static constexpr int OFF_PART = OFF_MISC + 16;              // float2 [NPB][2 sets][8][32]
   static constexpr int OFF_LSE = OFF_PART + NPB * 16 * 32 * 8; // float [NLB][128]
   static constexpr int OFF_MERGE = OFF_LSE + NLB * 128 * 4;   // float [MERGE_SEGS][128]
@@ -105,12 +105,15 @@ struct Smem {
   static constexpr int DYN_BYTES = TOTAL + 1024;            // slack for 1024-byte alignment
 };
 
-__device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity) {
+// Wait of the abort path (the abort flag is already set, so it is not looked at): for a copy
+// or an MMA that is in flight and will complete.
+__device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity,
+                                                unsigned long long limit_ns) {
   const unsigned long long t0 = globaltimer_ns();
   for (;;) {
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) return false;
+    if (globaltimer_ns() - t0 > limit_ns) return false;
   }
 }
 
@@ -126,7 +129,7 @@ __device__ __forceinline__ bool mbar_wait_warp_relaxed(uint32_t bar, uint32_t pa
     int stop = 0;
     if ((threadIdx.x & 31) == 0) {
       if (*abort_flag != 0) stop = 1;
-      else if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = code; stop = 1; }
+      else if (globaltimer_ns() - t0 > wait_limit_ns(abort_flag)) { *abort_flag = code; stop = 1; }
     }
     if (__shfl_sync(0xffffffffu, stop, 0)) return false;
   }
@@ -144,17 +147,17 @@ struct Item {
 };
 
 // CTA `c` of `G` owns tiles [c*TT/G, (c+1)*TT/G) of a phase's TT tiles.
-__device__ __forceinline__ long long part_lo(long long c, long long TT, int G) { return c * TT / G; }
+__host__ __device__ __forceinline__ long long part_lo(long long c, long long TT, int G) { return c * TT / G; }
 // the CTA whose range contains tile x: the largest c with part_lo(c) <= x
-__device__ __forceinline__ int cta_of_tile(long long x, long long TT, int G) {
+__host__ __device__ __forceinline__ int cta_of_tile(long long x, long long TT, int G) {
   return static_cast<int>(((x + 1) * G + TT - 1) / TT) - 1;
 }
 
 // Calls f(item) for every work item of this CTA in schedule order; stops when f
 // returns false.  All three warp roles walk the same list.
 template <typename F>
-__device__ __forceinline__ void for_each_item(const ScoreArgs& a, int cta, int G, int lag,
-                                              F&& f) {
+__host__ __device__ __forceinline__ void for_each_item(const ScoreArgs& a, int cta, int G, int lag,
+                                                       F&& f) {
   // Phase order: statistics run `lag` waves ahead of votes: S(0) .. S(lag-1) V(0) S(lag)
   // V(1) ...; lag = 1 is the plain order S(0) V(0) S(1) V(1) ...
   int s_next = a.votes_only ? a.nwaves : 0, v_next = 0;
@@ -163,7 +166,7 @@ __device__ __forceinline__ void for_each_item(const ScoreArgs& a, int cta, int G
     if (s_next < a.nwaves && s_next - v_next < lag) { w = s_next++; vote = 0; }
     else { w = v_next++; vote = 1; }
     const int u0 = w * a.upw;
-    const int nu = min(a.upw, a.units - u0);
+    const int nu = a.upw < a.units - u0 ? a.upw : a.units - u0;
     const int T = vote ? a.T2 : a.T1;
     const long long TT = static_cast<long long>(nu) * T;
     const long long lo = part_lo(cta, TT, G), hi = part_lo(cta + 1, TT, G);
@@ -172,7 +175,8 @@ __device__ __forceinline__ void for_each_item(const ScoreArgs& a, int cta, int G
       Item it;
       it.unit = u0 + ul;
       it.t0 = static_cast<int>(pos - static_cast<long long>(ul) * T);
-      it.t1 = static_cast<int>(min(static_cast<long long>(T), it.t0 + (hi - pos)));
+      const long long t1 = it.t0 + (hi - pos);
+      it.t1 = static_cast<int>(t1 < T ? t1 : T);
       it.vote = vote;
       // where this CTA's partial of the unit goes / how many partials the unit gets:
       // both follow from the statistics-pass partition of the unit's wave
@@ -262,6 +266,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     mbar_init(bar_drain, 1);
     mbar_init(bar_merge, 1);
     *abort_s = 0;
+    *reinterpret_cast<volatile unsigned long long*>(abort_s + 1) = a.wait_ns;
     mbar_fence_init();
   }
   if (warp == 1) {
@@ -335,12 +340,12 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         for (int b = 0; b < 2; ++b) {
           int last = -1;
           for (int i = b; i < nitem; i += 2) last = i;
-          if (last >= 0) mbar_wait_drain(bar_qf(b), (last >> 1) & 1);
+          if (last >= 0) mbar_wait_drain(bar_qf(b), (last >> 1) & 1, a.wait_ns);
         }
         for (int s = 0; s < STAGES; ++s) {
           int last = -1;
           for (int i = s; i < git; i += STAGES) last = i;
-          if (last >= 0) mbar_wait_drain(bar_full(s), (last / STAGES) & 1);
+          if (last >= 0) mbar_wait_drain(bar_full(s), (last / STAGES) & 1, a.wait_ns);
         }
       }
     }
@@ -397,7 +402,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
       });
       if (*abort_s != 0) {
         tc_commit(bar_drain);
-        mbar_wait_drain(bar_drain, 0);
+        mbar_wait_drain(bar_drain, 0, a.wait_ns);
       }
     }
   } else if (warp < 2 + EPI_WARPS || warp >= 4 + EPI_WARPS) {
@@ -581,10 +586,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     });
   } else {
     // ------------------------------------------------------------ book-keeper warps
-    // Warp 10 publishes this CTA's statistics partials (and merges a unit when it was the
-    // last to publish); warp 11 fetches the merged log-sum-exp rows the vote items need.
-    // Each walks its own kind of item in schedule order, so publishing never waits for
-    // another CTA and the fetcher runs as far ahead as its shared-memory buffers allow.
+    // Warp 10 publishes this CTA's statistics partials; warp 11 fetches the unit's partials
+    // for every vote item and folds them into the log-sum-exp row the item needs.  Each
+    // walks its own kind of item in schedule order, so publishing never waits for another
+    // CTA and the fetcher runs as far ahead as its shared-memory buffers allow.
     const bool publisher = warp == 2 + EPI_WARPS;  // warp 10; warp 11 is the fetcher
     int nstat = 0, nvote = 0, nmerge = 0;
     const float* merge_s = reinterpret_cast<const float*>(smem + SM::OFF_MERGE);
@@ -615,91 +620,86 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           a.partials[(static_cast<size_t>(it.unit) * a.maxseg + it.slot) * MAX_COLS + c] =
               M + log2f(S);
         }
+        // release: the partial is visible to whoever sees the count
         __threadfence();
         __syncwarp();
-        int last = 0;
         if (lane == 0) {
-          last = (atomicAdd(a.counters + it.unit, 1) == it.nseg - 1) ? 1 : 0;
+          atomicAdd(a.counters + it.unit, 1);
           mbar_arrive(bar_pe(pb));
-        }
-        if (__shfl_sync(0xffffffffu, last, 0)) {
-          // this was the unit's last partial: fold all of them, in slot order, into one
-          // -log2-sum-exp per window row, then raise the count once more to say so.  The
-          // unit's partials are contiguous: one bulk copy brings up to MERGE_SEGS of them
-          // into shared memory (a single trip through the loaded memory system instead of
-          // one per batch of register loads); each lane then owns four adjacent rows.
-          (void)ld_acquire(a.counters + it.unit);
-          fence_proxy_async();
-          const float* pp = a.partials + static_cast<size_t>(it.unit) * a.maxseg * MAX_COLS;
-          const int c4 = lane * 4;
-          float M[4], S[4];
-#pragma unroll
-          for (int t = 0; t < 4; ++t) { M[t] = -INFINITY; S[t] = 0.f; }
-          for (int s0 = 0; s0 < it.nseg; s0 += MERGE_SEGS, ++nmerge) {
-            const int ns = min(MERGE_SEGS, it.nseg - s0);
-            if (lane == 0) {
-              mbar_expect_tx(bar_merge, ns * MAX_COLS * 4);
-              bulk_load(sbase + SM::OFF_MERGE, pp + static_cast<size_t>(s0) * MAX_COLS,
-                        ns * MAX_COLS * 4, bar_merge);
-            }
-            if (!mbar_wait_warp_relaxed(bar_merge, nmerge & 1, abort_s, WAIT_MERGE_COPY)) {
-              mbar_wait_drain(bar_merge, nmerge & 1);  // never leave with the copy in flight
-              return false;
-            }
-            if (c4 < a.ncols) {
-              for (int sg = 0; sg < ns; ++sg) {
-                const float4 x = *reinterpret_cast<const float4*>(merge_s + sg * MAX_COLS + c4);
-                const float pv[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                  const float Mn = fmaxf(fmaxf(M[t], pv[t]), -1e30f);
-                  S[t] = S[t] * ex2_approx(M[t] - Mn) + ex2_approx(pv[t] - Mn);
-                  M[t] = Mn;
-                }
-              }
-            }
-            __syncwarp();  // all lanes are done with the buffer before the next copy lands
-          }
-          if (c4 < a.ncols) {
-            float4 out;
-            out.x = -(M[0] + log2f(S[0]));
-            out.y = -(M[1] + log2f(S[1]));
-            out.z = -(M[2] + log2f(S[2]));
-            out.w = -(M[3] + log2f(S[3]));
-            *reinterpret_cast<float4*>(a.lse2 + static_cast<size_t>(it.unit) * MAX_COLS + c4) = out;
-          }
-          __threadfence();
-          __syncwarp();
-          if (lane == 0) atomicAdd(a.counters + it.unit, 1);
         }
         ++nstat;
         return true;
       }
-      // the merged -log2-sum-exp of the unit's window rows goes into a shared-memory
-      // buffer as soon as the unit's count says it is ready (bounded wait) and the softmax
-      // warps are done with that buffer
+      // Fetcher.  A vote item needs minus the log2-sum-exp of every window row of its unit.
+      // With a supplied normaliser that row is in global memory already.  Otherwise it is
+      // the fold of the unit's partials: as soon as the unit's count says that all of them
+      // are published (bounded wait), this warp pulls them into shared memory with bulk
+      // copies (they are contiguous, 512 bytes each) and folds them in slot order, the same
+      // order in every CTA and every run, so all CTAs get bit-identical rows without a
+      // second hand-over through global memory.
       const int lb = nvote % NLB;
-      if (!mbar_wait_warp_relaxed(bar_le(lb), ((nvote / NLB) & 1) ^ 1, abort_s, WAIT_LSE_EMPTY))
-        return false;
+      const int ready = a.votes_only ? 0 : it.nseg - 1;  // count must exceed this
       int stop = 0;
-      if (lane == 0 && ld_acquire(a.counters + it.unit) <= it.nseg) {
+      if (lane == 0 && ld_acquire(a.counters + it.unit) <= ready) {
         const unsigned long long t0 = globaltimer_ns();
         for (;;) {
-          if (ld_acquire(a.counters + it.unit) > it.nseg) break;
+          if (ld_acquire(a.counters + it.unit) > ready) break;
           if (*abort_s != 0) { stop = 1; break; }
-          if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort_s = WAIT_UNIT_STATS; stop = 1; break; }
+          // half the limit: the roles of this CTA that wait for this row then still see the
+          // abort flag, not their own time-out, and the status names the wait that failed
+          if (globaltimer_ns() - t0 > a.wait_ns / 2) { *abort_s = WAIT_UNIT_STATS; stop = 1; break; }
           __nanosleep(100);
         }
       }
       if (__shfl_sync(0xffffffffu, stop, 0)) return false;
       (void)ld_acquire(a.counters + it.unit);  // every lane orders its reads after the count
-      {
-        const int c4 = lane * 4;
-        float4 val = make_float4(0.f, 0.f, 0.f, 0.f);
+      const int c4 = lane * 4;
+      float4 val = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (a.votes_only) {
         if (c4 < a.ncols)
           val = __ldcg(reinterpret_cast<const float4*>(a.lse2 + static_cast<size_t>(it.unit) * MAX_COLS + c4));
-        *reinterpret_cast<float4*>(lse_s + lb * MAX_COLS + c4) = val;
+      } else {
+        fence_proxy_async();
+        const float* pp = a.partials + static_cast<size_t>(it.unit) * a.maxseg * MAX_COLS;
+        float M[4], S[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) { M[t] = -INFINITY; S[t] = 0.f; }
+        for (int s0 = 0; s0 < it.nseg; s0 += MERGE_SEGS, ++nmerge) {
+          const int ns = min(MERGE_SEGS, it.nseg - s0);
+          if (lane == 0) {
+            mbar_expect_tx(bar_merge, ns * MAX_COLS * 4);
+            bulk_load(sbase + SM::OFF_MERGE, pp + static_cast<size_t>(s0) * MAX_COLS,
+                      ns * MAX_COLS * 4, bar_merge);
+          }
+          if (!mbar_wait_warp_relaxed(bar_merge, nmerge & 1, abort_s, WAIT_MERGE_COPY)) {
+            mbar_wait_drain(bar_merge, nmerge & 1, a.wait_ns);  // never leave with the copy in flight
+            return false;
+          }
+          if (c4 < a.ncols) {
+            for (int sg = 0; sg < ns; ++sg) {
+              const float4 x = *reinterpret_cast<const float4*>(merge_s + sg * MAX_COLS + c4);
+              const float pv[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+              for (int t = 0; t < 4; ++t) {
+                const float Mn = fmaxf(fmaxf(M[t], pv[t]), -1e30f);
+                S[t] = S[t] * ex2_approx(M[t] - Mn) + ex2_approx(pv[t] - Mn);
+                M[t] = Mn;
+              }
+            }
+          }
+          __syncwarp();  // all lanes are done with the buffer before the next copy lands
+        }
+        if (c4 < a.ncols) {
+          val.x = -(M[0] + log2f(S[0]));
+          val.y = -(M[1] + log2f(S[1]));
+          val.z = -(M[2] + log2f(S[2]));
+          val.w = -(M[3] + log2f(S[3]));
+        }
       }
+      // the softmax warps must be done with this buffer's previous row
+      if (!mbar_wait_warp_relaxed(bar_le(lb), ((nvote / NLB) & 1) ^ 1, abort_s, WAIT_LSE_EMPTY))
+        return false;
+      *reinterpret_cast<float4*>(lse_s + lb * MAX_COLS + c4) = val;
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_lf(lb));
       ++nvote;
@@ -815,6 +815,48 @@ cudaError_t run_scores(const CUtensorMap& tmK, const CUtensorMap& tmQ, const Sco
 
 }  // namespace
 
+// The part of the kernel's arguments that fixes the schedule (what for_each_item reads).
+static ScoreArgs schedule_args(const ScorePlan& plan, int L, int W, int Hkv, int votes_only) {
+  ScoreArgs a = {};
+  a.L = L;
+  a.n = L - W;
+  a.W = W;
+  a.Hkv = Hkv;
+  a.hpu = plan.hpu;
+  a.ncols = plan.ncols;
+  a.npad = plan.npad;
+  a.sub_per_kv = plan.sub_per_kv;
+  a.g = plan.g;
+  a.units = plan.units;
+  a.upw = plan.units_per_wave;
+  a.nwaves = plan.nwaves;
+  a.T1 = plan.tiles_stats;
+  a.T2 = plan.tiles_vote;
+  a.maxseg = plan.maxseg;
+  a.pipelined = plan.pipelined;
+  a.votes_only = votes_only;
+  if (votes_only) {  // nothing couples the units any more: one phase over all of them
+    a.upw = plan.units;
+    a.nwaves = 1;
+  }
+  return a;
+}
+
+int list_schedule_items(const ScorePlan& plan, int L, int W, int Hkv, int votes_only, int grid,
+                        int cta, int32_t* out, int max_items) {
+  const ScoreArgs a = schedule_args(plan, L, W, Hkv, votes_only);
+  int count = 0;
+  for_each_item(a, cta, grid, a.pipelined, [&](const Item& it) {
+    if (count < max_items) {
+      int32_t* o = out + static_cast<size_t>(count) * 6;
+      o[0] = it.unit; o[1] = it.t0; o[2] = it.t1; o[3] = it.vote; o[4] = it.slot; o[5] = it.nseg;
+    }
+    ++count;
+    return true;
+  });
+  return count;
+}
+
 bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* plan) {
   if (B < 1 || Hq < 1 || Hkv < 1 || L < 1 || W < 1 || W > L || Hq % Hkv != 0) return false;
   if (W > MAX_COLS || (d != 64 && d != 128)) return false;
@@ -869,7 +911,8 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrid
                                  int Hq, int Hkv, int L, int d, int W, const ScorePlan& plan,
                                  float* vote, int* status,
                                  int* counters, float* partials, float* lse2, cudaStream_t stream,
-                                 int* launches, const float* lse_obs, bool keep_status) {
+                                 int* launches, const float* lse_obs, bool keep_status,
+                                 bool never_ready) {
   CUtensorMap tmK, tmQ;
   {
     // (d, position, KV head, batch) with the caller's strides: any layout whose rows of d
@@ -887,28 +930,8 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrid
     cuuint32_t box[2] = {64, static_cast<cuuint32_t>(plan.npad)};
     if (!encode_map(&tmQ, q_obs, 2, dims, strides, box)) return cudaErrorInvalidValue;
   }
-  ScoreArgs a;
-  a.L = L;
-  a.n = L - W;
-  a.W = W;
-  a.Hkv = Hkv;
-  a.hpu = plan.hpu;
-  a.ncols = plan.ncols;
-  a.npad = plan.npad;
-  a.sub_per_kv = plan.sub_per_kv;
-  a.g = plan.g;
-  a.units = plan.units;
-  a.upw = plan.units_per_wave;
-  a.nwaves = plan.nwaves;
-  a.T1 = plan.tiles_stats;
-  a.T2 = plan.tiles_vote;
-  a.maxseg = plan.maxseg;
-  a.pipelined = plan.pipelined;
-  a.votes_only = lse_obs ? 1 : 0;
-  if (lse_obs) {  // nothing couples the units any more: one phase over all of them
-    a.upw = plan.units;
-    a.nwaves = 1;
-  }
+  ScoreArgs a = schedule_args(plan, L, W, Hkv, (lse_obs || never_ready) ? 1 : 0);
+  a.wait_ns = wait_limit_setting();
   a.c2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
   a.partials = partials;
   a.lse2 = lse2;

@@ -360,6 +360,42 @@ def test_full_size_workloads_on_sampled_heads(wid, layer, budget, nheads):
     _check_compress(None, w.W, w.pool_kernel, w.pool_type, budget, heads=heads, dev=dev)
 
 
+@pytest.mark.parametrize("wid,layer,heads", [
+    # workload 2 (the benchmarked shape): heads in different batches, i.e. in different waves
+    # of the scoring schedule, and all four heads of one KV group once
+    (2, 0, [(0, 0), (0, 31), (1, 9), (2, 18), (3, 4), (3, 5), (3, 6), (3, 7)]),
+    (2, 17, [(0, 12), (1, 30), (2, 1), (3, 23)]),
+    # workload 3: W = 64, two head sub-groups per KV head (column-split epilogue)
+    (3, 0, [(0, 0), (0, 2), (0, 15), (0, 29)]),
+])
+def test_full_size_votes_of_the_recomputing_path(wid, layer, heads):
+    """Eq. 1 element by element at full size: every vote of the sampled heads, from the
+    two-sweep scoring call in the configuration the benchmark times."""
+    w = synth.WORKLOADS[wid]
+    dev = synth.make_layer(w, layer, device="cuda", want_v=False)
+    vote, ws = sk.snapkv_window_scores(dev["q_obs"], dev["k"])
+    code, detail = sk.snapkv_device_status(ws)
+    assert code == sk.OK, (code, detail)
+    qb, kb = _bits(dev["q_obs"]), _bits(dev["k"])
+    worst = 0.0
+    for b, h in heads:
+        ref = _oracle_head(qb, kb, b, h, w.Hq // w.Hkv)
+        worst = max(worst, parity.check_votes(vote[b, h].cpu().numpy(), ref))
+    assert worst < 1e-4  # fp32 accumulation and exp2.approx leave about 1e-6
+
+
+def test_fused_call_leaves_the_same_votes_as_the_staged_call():
+    # the whole-step entry point scores into its workspace; what it selects from must be the
+    # votes the staged scoring call returns, bit for bit (same kernel, same schedule)
+    w = synth.WORKLOADS[2]
+    dev = synth.make_layer(w, 5, device="cuda")
+    budget = w.budgets[-1]
+    ok, ov, oi, ws = sk.snapkv_compress(dev["q_obs"], dev["k"], dev["v"], w.pool_kernel, PT[w.pool_type], budget)
+    staged, _ = sk.snapkv_window_scores(dev["q_obs"], dev["k"])
+    idx = sk.snapkv_pool_topk(staged.view(w.B * w.Hq, w.n), w.pool_kernel, PT[w.pool_type], budget - w.W)
+    assert torch.equal(idx.view_as(oi), oi)
+
+
 def test_extreme_prompt_keeps_the_needle():
     w = synth.WORKLOADS[4]
     dev = synth.make_layer(w, 0, device="cuda")
