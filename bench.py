@@ -26,8 +26,29 @@ if ROOT not in sys.path:
 import torch  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries
-# (profiles/): (stage, workload id) -> bytes; None for anything not captured
-NCU_TRAFFIC = {("score", 2): 464.6e6, ("gather", 2): 338.7e6, ("score-lse", 2): 275.9e6}
+# (profiles/): (stage, workload id) -> (bytes, source file of the kernel, first 12 hex digits of
+# that file's SHA-256 when the counters were taken).  A figure is reported only while the
+# kernel's source is unchanged; after any edit it reads null until the capture is redone.
+NCU_TRAFFIC = {
+    ("score", 2): (464.6e6, "snapkv_score.cu", "unset"),
+    ("score-lse", 2): (275.9e6, "snapkv_score.cu", "unset"),
+    ("gather", 2): (338.7e6, "snapkv_gather.cu", "unset"),
+}
+
+
+def ncu_traffic(stage, wid):
+    import hashlib
+    ent = NCU_TRAFFIC.get((stage, wid))
+    if ent is None:
+        return None
+    nbytes, src, digest = ent
+    path = os.path.join(ROOT, "paper_2404_14469_b200", "csrc", src)
+    try:
+        with open(path, "rb") as f:
+            now = hashlib.sha256(f.read()).hexdigest()[:12]
+    except OSError:
+        return None
+    return nbytes if now == digest else None
 
 METRIC = "prompt_tokens_compressed_per_s"
 UNIT = "prompt tokens/s"
@@ -150,19 +171,26 @@ def oracle_sample(w, budget, seconds_hint=15.0):
 def run_reference(args, w, budget, rank, world):
     if rank != 0:
         return
-    vals = []
+    vals, times = [], []
     desc, cores = "", 0
     for _ in range(args.warmup + args.steps):
-        tps, cores, desc, _ = oracle_sample(w, budget, seconds_hint=8.0)
+        tps, cores, desc, t_sample = oracle_sample(w, budget, seconds_hint=8.0)
         vals.append(tps)
+        times.append(t_sample)
     vals = vals[args.warmup:] or vals
+    times = times[args.warmup:] or times
     value = sum(vals) / len(vals)
-    ms_step = w.B * w.L / value * 1e3
+    # a step of this arm is a bounded sample of the workload: ms_per_step is the time one such
+    # sample really took; what the whole 32-layer step would take is given separately
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sum(times) / len(times) * 1e3,
+        "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": workload_config(w, budget, args.layers or w.layers),
+        "extrapolated": {"ms_per_full_step": w.B * w.L / value * 1e3,
+                         "note": "value and ms_per_full_step scale the sampled (batch, head) rows "
+                                 "to the whole layer stack; ms_per_step is the sample itself"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -174,6 +202,19 @@ def workload_config(w, budget, layers):
     return {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "d": w.d, "L": w.L, "W": w.W,
             "pool": f"{w.pool_type}{w.pool_kernel}", "budget": budget, "layers": layers,
             "l2": "every layer has its own buffers (inputs per step far larger than L2)"}
+
+
+def launch_ranks(n, argv):
+    """`python bench.py --gpus N` outside a launcher: run N ranks of this script through
+    torch.distributed.run on 127.0.0.1 (one process per GPU) and pass their exit code on."""
+    import socket
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
 
 
 # ------------------------------------------------------------------ our arm
@@ -195,6 +236,10 @@ def main():
                     help="time the shared-selection variant (snapkv_compress_grouped): one "
                          "selection per KV head, the compressed cache keeps Hkv heads")
     args = ap.parse_args()
+
+    if args.gpus > 1 and "RANK" not in os.environ:
+        # not under a launcher: start one rank per GPU ourselves, the way the launcher would
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
 
     from paper_2404_14469_b200 import synth
 
@@ -267,7 +312,12 @@ def main():
     torch.cuda.synchronize()
     barrier(world)
 
-    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local)
+    # nvidia-smi numbers the GPUs of the machine, CUDA those this process may see: go by UUID
+    try:
+        smi_id = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:
+        smi_id = str(local)
+    sampler = ClockSampler(smi_id)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
@@ -353,7 +403,7 @@ def main():
                                     "gather": "gather_kernel"}[dom],
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
         "peak_kind": f"of {peak_kind}",
-        "traffic": NCU_TRAFFIC.get(("score-lse" if args.lse_in and dom == "score" else dom, w.wid)),
+        "traffic": ncu_traffic("score-lse" if args.lse_in and dom == "score" else dom, w.wid),
         "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": stage_ms[dom],
         "stage_ms_per_layer": stage_ms,
         "whole_step": {"algorithmic_bytes_per_layer": ab["total"], "ms_per_layer": ms_layer,
@@ -402,8 +452,6 @@ def main():
 
     if rank == 0:
         cfg = workload_config(w, budget, layers)
-        cfg["ms_per_layer"] = ms_layer
-        cfg["parallelism"] = "replicas: each GPU compresses its own batch, no collective"
         if args.lse_in:
             cfg["variant"] = ("lse-in: the window rows' log-sum-exp is an input, one sweep over K "
                               "(snapkv_compress_lse; not the paper's path)")
@@ -414,7 +462,10 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "dtype_note": "bf16 operands on the tensor cores, fp32 accumulation, softmax and votes",
+            "ms_per_layer": ms_layer,
+            "parallelism": "replicas: each GPU compresses its own batch, no collective",
             "config": cfg, "clocks": clocks, "e2e": e2e,
             "gpu_launches": launches_per_layer * layers * args.steps,
             "roofline": roofline, "cpu_baseline": cpu_baseline,

@@ -14,7 +14,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsnapkv.so")
 SOURCES = ["snapkv_api.cu", "snapkv_score.cu", "snapkv_select.cu", "snapkv_gather.cu",
            "snapkv_metrics.cu", "snapkv_decode.cu"]
-HEADERS = ["sm100_ptx.cuh", "snapkv_internal.h", os.path.join("..", "..", "include", "snapkv.h")]
+HEADERS = ["sm100_ptx.cuh", "snapkv_internal.h", "launch.cuh", os.path.join("..", "..", "include", "snapkv.h")]
 
 
 def _nvcc() -> str:
@@ -39,7 +39,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [
         _nvcc(), "-shared", "-o", LIB,
         "-gencode", "arch=compute_100a,code=sm_100a",
-        "-O3", "-std=c++17", "-lineinfo",
+        "-O3", "-std=c++17", "-lineinfo", "--expt-relaxed-constexpr",
         "-Xcompiler", "-fPIC,-O3,-Wall",
         "-cudart", "static",
     ]

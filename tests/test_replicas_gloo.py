@@ -59,3 +59,23 @@ def test_single_process_defaults():
     assert replicas.env_rank_world() == (0, 1, 0)
     assert replicas.max_over_ranks(3.5, 1) == 3.5
     assert replicas.aggregate_throughput(100, 1, 10.0) == 10000.0
+
+
+def test_bench_launches_its_own_ranks_when_asked_for_two_gpus():
+    # `bench.py --gpus 2` outside a launcher starts two ranks itself.  The reference arm needs
+    # no GPU: rank 0 times the oracle on a small sample and prints the line, rank 1 exits 0.
+    import json
+    import subprocess
+
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference",
+                          "--workload", "0", "--steps", "1", "--warmup", "0"],
+                         capture_output=True, text=True, timeout=600, env=env, cwd=ROOT)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(x) for x in res.stdout.splitlines() if x.startswith("{")]
+    assert len(lines) == 1                       # one line for the whole job, from rank 0
+    line = lines[0]
+    assert line["impl"] == "reference" and line["n_gpus"] == 2
+    assert line["config"]["workload"] == "tiny-1k" or line["config"]["L"] == 1024
+    assert line["value"] > 0 and line["cpu_baseline"]["kind"] == "oracle"
+    assert line["extrapolated"]["ms_per_full_step"] > 0
