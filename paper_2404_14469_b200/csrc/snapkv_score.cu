@@ -46,10 +46,7 @@ namespace snapkv {
 
 namespace {
 
-#ifndef SNAPKV_STAGES
-#define SNAPKV_STAGES 4
-#endif
-constexpr int STAGES = SNAPKV_STAGES;
+constexpr int STAGES = 4;
 constexpr int NBUF = 4;               // TMEM accumulator buffers of 128 columns
 constexpr int TMEM_COLS = 512;
 constexpr int SUBTILE_BYTES = 128 * 128;  // 128 rows x 64 bf16, 128-byte swizzled
@@ -57,12 +54,6 @@ constexpr int EPI_WARPS = 8;           // softmax warps per set (two warpgroups)
 // Warps: 0 producer, 1 MMA issuer, 2-9 softmax set 0, 10 publisher, 11 lse fetcher and, in
 // split mode, 12-19 softmax set 1.
 constexpr int threads_for(bool split) { return split ? 640 : 384; }
-#ifndef SNAPKV_L2_PREFETCH
-#define SNAPKV_L2_PREFETCH 0
-#endif
-#ifndef SNAPKV_V_LD16
-#define SNAPKV_V_LD16 0
-#endif
 #ifndef WAVE_MIB
 #define WAVE_MIB 64
 #endif
@@ -327,21 +318,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         ++nitem;
         const int kb = ukv / a.Hkv, kh = ukv - kb * a.Hkv;  // the K map is (d, L, Hkv, B)
         const int nt = it.t1 - it.t0;
-#if SNAPKV_L2_PREFETCH > 0
-        // tiles STAGES .. PREFETCH-1 of the item: their ring slots are not free yet, but their
-        // trip from HBM to L2 can start now
-        for (int k = STAGES; k < SNAPKV_L2_PREFETCH && k < nt; ++k)
-          for (int sb = 0; sb < SUBT; ++sb)
-            tma_prefetch_l2_4d(&tmK, sb * 64, tile_of(it, k) * TILE_KEYS, kh, kb);
-#endif
         for (int k = 0; k < nt; ++k, ++git) {
           const int s = git % STAGES;
           const uint32_t ph = (git / STAGES) & 1;
-#if SNAPKV_L2_PREFETCH > 0
-          if (k + SNAPKV_L2_PREFETCH < nt)
-            for (int sb = 0; sb < SUBT; ++sb)
-              tma_prefetch_l2_4d(&tmK, sb * 64, tile_of(it, k + SNAPKV_L2_PREFETCH) * TILE_KEYS, kh, kb);
-#endif
           if (!mbar_wait_thread(bar_empty(s), ph ^ 1, abort_s, WAIT_PRODUCER_EMPTY)) return false;
           mbar_expect_tx(bar_full(s), SM::STAGE_BYTES);
           const int key0 = tile_of(it, k) * TILE_KEYS;
@@ -385,6 +364,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         const int qb = nitem & 1;
         if (!mbar_wait_thread(bar_qf(qb), (nitem >> 1) & 1, abort_s, WAIT_Q_FULL)) return false;
         ++nitem;
+        const uint64_t qd0 = umma_desc_k128(q_s(qb));
         const int nt = it.t1 - it.t0;
         for (int k = 0; k < nt;) {
           const int s = git % STAGES;
@@ -400,15 +380,29 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * 128;
+          // One descriptor per operand and tile; the eight K-slices of the tile differ from it
+          // by constants (the start-address field counts 16-byte units and the operands sit
+          // below 256 KB, so adding to the low word never carries into another field).  The
+          // issuing thread is a single in-order instruction stream: every instruction saved
+          // per tcgen05.mma shortens the time between two of them.
+          const uint64_t kd0 = umma_desc_k128(stage_addr(s, 0));
+          constexpr uint64_t K_SB = (2 * SUBTILE_BYTES) >> 4;  // next 64 elements of d (stage pairs interleave)
+          constexpr uint64_t Q_SB = SUBTILE_BYTES >> 4;
+          if (it.vote) {
 #pragma unroll
-          for (int sb = 0; sb < SUBT; ++sb) {
+            for (int sb = 0; sb < SUBT; ++sb)
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-              const uint64_t kd = umma_desc_k128(stage_addr(s, sb) + kk * 32);
-              const uint64_t qd = umma_desc_k128(q_s(qb) + sb * SUBTILE_BYTES + kk * 32);
-              if (it.vote) tc_mma_bf16(d_tmem, kd, qd, idesc_v, (sb | kk) != 0);
-              else tc_mma_bf16(d_tmem, qd, kd, pair ? idesc_s2 : idesc_s, (sb | kk) != 0);
-            }
+              for (int kk = 0; kk < 4; ++kk)
+                tc_mma_bf16(d_tmem, kd0 + (sb * K_SB + kk * 2), qd0 + (sb * Q_SB + kk * 2), idesc_v,
+                            (sb | kk) != 0);
+          } else {
+            const uint32_t idesc = pair ? idesc_s2 : idesc_s;
+#pragma unroll
+            for (int sb = 0; sb < SUBT; ++sb)
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk)
+                tc_mma_bf16(d_tmem, qd0 + (sb * Q_SB + kk * 2), kd0 + (sb * K_SB + kk * 2), idesc,
+                            (sb | kk) != 0);
           }
           tc_commit(bar_empty(s));
           if (pair) tc_commit(bar_empty(s + 1));
@@ -539,41 +533,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           __syncwarp();
           if (lane == 0) mbar_arrive_n(bar_te(buf), te_arrivals);
         }
-#if SNAPKV_V_LD16
-        if (SPLIT) {
-          // 16 columns at a time, the next group's TMEM read in flight while this one is
-          // turned into probabilities
-          float v2[2][16];
-          tmem_ld16(taddr, v2[0]);
-#pragma unroll
-          for (int gi = 0; gi < VCH * 2; ++gi) {
-            tmem_wait_ld();
-            if (gi + 1 < VCH * 2) {
-              tmem_ld16(taddr + (gi + 1) * 16, v2[(gi + 1) & 1]);
-            } else {
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) mbar_arrive_n(bar_te(buf), te_arrivals);
-            }
-            const float(&vc)[16] = v2[gi & 1];
-            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-            for (int t4 = 0; t4 < 4; ++t4) {
-              const float4 z = *reinterpret_cast<const float4*>(lse_b + coff + gi * 16 + 4 * t4);
-              a0 += ex2_approx(fmaf(vc[4 * t4 + 0], a.c2, z.x));
-              a1 += ex2_approx(fmaf(vc[4 * t4 + 1], a.c2, z.y));
-              a2 += ex2_approx(fmaf(vc[4 * t4 + 2], a.c2, z.z));
-              a3 += ex2_approx(fmaf(vc[4 * t4 + 3], a.c2, z.w));
-            }
-            g16[gi] = (a0 + a1) + (a2 + a3);
-          }
-        }
         if (SPLIT || w16) {
-          if (!SPLIT) {
-#else
-        if (SPLIT || w16) {
-          {
-#endif
 #pragma unroll
           for (int ch = 0; ch < VCH; ++ch) {
             if (SPLIT) {
@@ -601,7 +561,6 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
               }
               g16[ch * 2 + hf] = (a0 + a1) + (a2 + a3);
             }
-          }
           }
           int hl = coff / a.W, left = gpw;  // SPLIT: coff is a multiple of W
           float acc = 0.f;
