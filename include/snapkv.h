@@ -335,6 +335,39 @@ snapkv_status_t snapkv_decode_attention(const void* q_cur, const void* cache_k, 
 snapkv_status_t snapkv_device_status(const void* workspace, void* stream, int* detail);
 
 /*
+ * The step on a PAGED cache (Listing 1 takes dense key_states / value_states; serving
+ * stacks keep the prompt's K and V in fixed-size pages of a shared pool and a per-sequence
+ * block table).  Position p of sequence b is row p % page_size of page
+ * page_table[b * pages_per_seq + p / page_size].
+ *   k_pool, v_pool  bf16, device: the pools.  Addressed as [page][KV head][row][d] with
+ *                   element strides k_strides[3] = {page, KV head, row} (v_strides likewise);
+ *                   rows of d elements contiguous, strides positive multiples of 8 elements,
+ *                   e.g. {Hkv*page_size*d, page_size*d, d} or {page_size*Hkv*d, d, Hkv*d}.
+ *   page_table      int32, device, [B][pages_per_seq].  Entries of pages a sequence does
+ *                   not reach are never read; an entry outside [0, num_pages) reads as
+ *                   zeros.  Pages may be shared between sequences (common prefixes).
+ *   page_size       positions per page: a multiple of 128, so that a tile of 128 keys lies in
+ *                   one page (SNAPKV_ERR_INVALID_ARG otherwise); pages_per_seq * page_size >= L.
+ *   seq_lens        host int32[B] or NULL.  NULL: every sequence has L positions.  Otherwise
+ *                   sequence b has seq_lens[b] in [W, L] positions and the call runs one
+ *                   single-sequence step per prompt (as snapkv_compress_varlen does), a
+ *                   sequence with budget >= its length being copied through.
+ *   lse_obs         optional, as in snapkv_compress_lse.
+ * What lies in a page behind a sequence's last position is never used (it may be anything).
+ * Outputs and workspace as for snapkv_compress (with seq_lens: as for
+ * snapkv_compress_varlen; the workspace must hold snapkv_workspace_size(1, Hq, Hkv, L_b, ...)
+ * of the longest sequence).  Results are bit-identical to snapkv_compress on a dense copy.
+ */
+snapkv_status_t snapkv_compress_paged(const void* q_obs, const void* k_pool, const void* v_pool,
+                                      const int64_t* k_strides, const int64_t* v_strides,
+                                      const int32_t* page_table, int pages_per_seq, int page_size,
+                                      int num_pages, const int32_t* seq_lens, const float* lse_obs,
+                                      int B, int Hq, int Hkv, int L, int d, int W,
+                                      int pool_kernel, int pool_type, int budget,
+                                      void* out_k, void* out_v, int32_t* out_idx,
+                                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The scoring kernel's schedule, for inspection (no counterpart in the paper).  The kernel
  * is a persistent grid; every block walks a fixed list of work items - tiles [t0, t1) of 128
  * keys of one unit (a batch, a KV head and up to 128 window columns of its query heads), in

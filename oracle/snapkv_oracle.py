@@ -36,6 +36,11 @@ A second one, for grouped-query attention: group_votes / compress_grouped let th
 heads of a group select TOGETHER on the KV head they share (Eq. 1's sum runs over the
 window rows of all the group's heads), which keeps the compressed cache at Hkv heads.
 
+read_paged / compress_paged read K and V through a block table (a paged cache: position p of
+sequence b is row p % page_size of page table[b][p // page_size] of a pool), one element row
+at a time, and then run the very same step: paging changes where a row lives, not what the
+method computes.
+
 hit_counts / hit_rate state the paper's hit-rate measure of a selection (Sec. 3, Eq. 3-7);
 decode_attention is the generation step's attention over the compressed cache (Sec. 5.1.2).
 
@@ -351,6 +356,36 @@ def compress_grouped(q_obs: np.ndarray, k: np.ndarray, v: np.ndarray, pool_kerne
             out_k[b, c, ksel:] = k[b, c, n:]
             out_v[b, c, ksel:] = v[b, c, n:]
     return {"out_k": out_k, "out_v": out_v, "out_idx": out_idx, "vote": vote, "pooled": pooled}
+
+
+def read_paged(pool: np.ndarray, table_row, page_size: int, length: int) -> np.ndarray:
+    """The first `length` positions of one sequence of a paged cache as a dense
+    [Hkv, length, d] array.  pool: [num_pages, Hkv, page_size, d]; table_row: page numbers."""
+    num_pages, Hkv, ps, d = pool.shape
+    assert ps == page_size
+    out = np.empty((Hkv, length, d), dtype=pool.dtype)
+    for p in range(length):
+        page = int(table_row[p // page_size])
+        if 0 <= page < num_pages:
+            out[:, p, :] = pool[page, :, p % page_size, :]
+        else:
+            out[:, p, :] = 0      # an entry that names no page of the pool reads as zeros
+    return out
+
+
+def compress_paged(q_obs: np.ndarray, k_pool: np.ndarray, v_pool: np.ndarray, page_table,
+                   page_size: int, seq_lens, pool_kernel: int, pool_type: int, budget: int,
+                   lse=None):
+    """Listing 1 per sequence on a paged cache.  q_obs [B, Hq, W, d]; pools
+    [num_pages, Hkv, page_size, d] (bf16 bit patterns); page_table [B, pages_per_seq];
+    seq_lens: B prompt lengths.  Returns one `compress` result per sequence."""
+    results = []
+    for b, length in enumerate(seq_lens):
+        k = read_paged(k_pool, page_table[b], page_size, int(length))[None]
+        v = read_paged(v_pool, page_table[b], page_size, int(length))[None]
+        results.append(compress(q_obs[b:b + 1], k, v, pool_kernel, pool_type, budget,
+                                lse=None if lse is None else lse[b:b + 1]))
+    return results
 
 
 def hit_counts(a_cur: np.ndarray, idx: np.ndarray, theta) -> np.ndarray:

@@ -29,6 +29,7 @@ SYMBOLS = [
     "snapkv_compress_grouped", "snapkv_compress_varlen",
     "snapkv_hit_counts", "snapkv_decode_workspace_size", "snapkv_decode_attention",
     "snapkv_set_wait_limit_ns", "snapkv_selftest_stalled_scores", "snapkv_schedule_items",
+    "snapkv_compress_paged",
 ]
 
 _lib = None
@@ -72,6 +73,9 @@ def lib() -> ctypes.CDLL:
     L.snapkv_compress_varlen.restype = c_int
     L.snapkv_compress_varlen.argtypes = ([c_vp] * 3 + [p64] * 4 + [p32, c_vp] + [c_int] * 9 + [c_vp] * 3
                                          + [c_vp, c_sz, c_vp])
+    L.snapkv_compress_paged.restype = c_int
+    L.snapkv_compress_paged.argtypes = ([c_vp] * 3 + [p64] * 2 + [c_vp] + [c_int] * 3 + [p32, c_vp]
+                                        + [c_int] * 9 + [c_vp] * 3 + [c_vp, c_sz, c_vp])
     L.snapkv_hit_counts.restype = c_int
     L.snapkv_hit_counts.argtypes = [c_vp, c_vp, c_int, c_int, c_int, ctypes.c_float, c_vp, c_vp]
     L.snapkv_decode_workspace_size.restype = c_sz
@@ -265,6 +269,53 @@ def snapkv_compress_varlen(q_obs, k, v, seq_lens, pool_kernel: int, pool_type: i
         pool_kernel, pool_type, budget, out_k.data_ptr(), out_v.data_ptr(), out_idx.data_ptr(),
         workspace.data_ptr(), workspace.numel(), _stream_ptr())
     _check(code, "snapkv_compress_varlen")
+    return out_k, out_v, out_idx, workspace
+
+
+def snapkv_compress_paged(q_obs, k_pool, v_pool, page_table, L, pool_kernel: int, pool_type: int,
+                          budget: int, seq_lens=None, lse_obs=None, workspace=None):
+    """The step on a paged cache.  k_pool, v_pool: bf16 CUDA views [num_pages, Hkv, page_size, d]
+    with contiguous rows (any other strides, e.g. a permuted [num_pages, page_size, Hkv, d]
+    pool); page_table: int32 CUDA [B, pages_per_seq]; L: prompt length (the longest one when
+    seq_lens, a list of B lengths, is given).  Returns (out_k, out_v, out_idx, workspace) as
+    snapkv_compress does, or, with seq_lens, as snapkv_compress_varlen does."""
+    _dev_bf16(q_obs, "q_obs"), _dev_bf16_rows(k_pool, "k_pool"), _dev_bf16_rows(v_pool, "v_pool")
+    if not (page_table.is_cuda and page_table.dtype == torch.int32 and page_table.is_contiguous()
+            and page_table.dim() == 2 and page_table.shape[0] == q_obs.shape[0]):
+        raise SnapKVError("page_table must be a contiguous CUDA int32 [B, pages_per_seq] tensor")
+    if tuple(v_pool.shape) != tuple(k_pool.shape):
+        raise SnapKVError("k_pool and v_pool must have the same shape")
+    B, Hq, W, d = q_obs.shape
+    num_pages, Hkv, page_size, dk = k_pool.shape
+    if dk != d:
+        raise SnapKVError("q_obs and k_pool disagree on the head dimension")
+    L_ = lib()
+    dev = k_pool.device
+    st = ctypes.c_int64 * 3
+    if seq_lens is None:
+        rows = L_.snapkv_out_rows(L, budget)
+        out_k = torch.empty(B, Hq, rows, d, dtype=torch.bfloat16, device=dev)
+        out_v = torch.empty_like(out_k)
+        out_idx = torch.empty(B, Hq, rows - W, dtype=torch.int32, device=dev)
+        eff_budget, lens_arg = rows, None
+        need = L_.snapkv_workspace_size(B, Hq, Hkv, L, d, W, pool_kernel, pool_type, eff_budget)
+    else:
+        lens = [int(x) for x in seq_lens]
+        out_k = torch.zeros(B, Hq, budget, d, dtype=torch.bfloat16, device=dev)
+        out_v = torch.zeros_like(out_k)
+        out_idx = torch.full((B, Hq, budget - W), -1, dtype=torch.int32, device=dev)
+        eff_budget, lens_arg = budget, (ctypes.c_int32 * B)(*lens)
+        need = max([L_.snapkv_workspace_size(1, Hq, Hkv, x, d, W, pool_kernel, pool_type, budget)
+                    for x in set(lens) if x > budget] + [256])
+    if workspace is None or workspace.numel() < need:
+        workspace = _alloc_ws(need, dev)
+    code = L_.snapkv_compress_paged(
+        q_obs.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(), st(*k_pool.stride()[:3]),
+        st(*v_pool.stride()[:3]), page_table.data_ptr(), page_table.shape[1], page_size, num_pages,
+        lens_arg, None if lse_obs is None else _lse_arg(lse_obs, B, Hq, W), B, Hq, Hkv, L, d, W,
+        pool_kernel, pool_type, eff_budget, out_k.data_ptr(), out_v.data_ptr(), out_idx.data_ptr(),
+        workspace.data_ptr(), workspace.numel(), _stream_ptr())
+    _check(code, "snapkv_compress_paged")
     return out_k, out_v, out_idx, workspace
 
 

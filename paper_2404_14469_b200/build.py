@@ -12,7 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsnapkv.so")
-SOURCES = ["snapkv_api.cu", "snapkv_score.cu", "snapkv_select.cu", "snapkv_gather.cu",
+SOURCES = ["snapkv_api.cu", "snapkv_score.cu", "snapkv_select.cu", "snapkv_select_cluster.cu", "snapkv_gather.cu",
            "snapkv_metrics.cu", "snapkv_decode.cu"]
 HEADERS = ["sm100_ptx.cuh", "snapkv_internal.h", "launch.cuh", os.path.join("..", "..", "include", "snapkv.h")]
 

@@ -246,7 +246,8 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
                                      void* workspace, size_t workspace_bytes, void* stream,
                                      bool keep_status, const float* lse_obs = nullptr,
                                      const KVStrides* k_str = nullptr,
-                                     const KVStrides* v_str = nullptr, bool grouped = false) {
+                                     const KVStrides* v_str = nullptr, bool grouped = false,
+                                     const PagedKV* paged = nullptr) {
   snapkv_status_t st = check_common(B, Hq, Hkv, L, d, W);
   if (st != SNAPKV_OK) return st;
   st = check_pool(pool_kernel, pool_type);
@@ -270,7 +271,7 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
     if (launch_iota_idx(out_idx, B * Ho, n, budget - W, s, &launches) != cudaSuccess)
       return SNAPKV_ERR_CUDA;
     if (launch_gather(k, v, ks, vs, nullptr, B, Ho, Hkv, L, d, W, n, budget, out_k, out_v, s,
-                      &launches) != cudaSuccess)
+                      &launches, paged) != cudaSuccess)
       return SNAPKV_ERR_CUDA;
     // no kernel of this path can time out, but a caller that passes a workspace may read its
     // status afterwards: it must not find what an earlier use of the memory left there
@@ -297,14 +298,14 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
                            reinterpret_cast<int*>(ws + w.off_counters),
                            reinterpret_cast<float*>(ws + w.off_partials),
                            reinterpret_cast<float*>(ws + w.off_lse), s, &launches, lse_obs,
-                           keep_status) != cudaSuccess)
+                           keep_status, false, paged) != cudaSuccess)
     return SNAPKV_ERR_CUDA;
   if (launch_pool_topk(vote, B * Ho, n, pool_kernel, pool_type, ksel, out_idx,
                        scratch ? reinterpret_cast<float*>(ws + w.off_pooled) : nullptr, s,
                        &launches, gsum) != cudaSuccess)
     return SNAPKV_ERR_CUDA;
   if (launch_gather(k, v, ks, vs, out_idx, B, Ho, Hkv, L, d, W, ksel, budget, out_k, out_v, s,
-                    &launches) != cudaSuccess)
+                    &launches, paged) != cudaSuccess)
     return SNAPKV_ERR_CUDA;
   g_last_launches = launches;
   return SNAPKV_OK;
@@ -425,6 +426,71 @@ snapkv_status_t snapkv_compress_varlen(const void* q_obs, const void* k, const v
                        out_idx ? out_idx + static_cast<size_t>(b) * Hq * (budget - W) : nullptr,
                        workspace, workspace_bytes, stream, /*keep_status=*/true,
                        lse_obs ? lse_obs + static_cast<size_t>(b) * Hq * W : nullptr, &ks, &vs);
+    if (st != SNAPKV_OK) return st;
+    launches += g_last_launches;
+  }
+  g_last_launches = launches;
+  return SNAPKV_OK;
+}
+
+snapkv_status_t snapkv_compress_paged(const void* q_obs, const void* k_pool, const void* v_pool,
+                                      const int64_t* k_strides, const int64_t* v_strides,
+                                      const int32_t* page_table, int pages_per_seq, int page_size,
+                                      int num_pages, const int32_t* seq_lens, const float* lse_obs,
+                                      int B, int Hq, int Hkv, int L, int d, int W, int pool_kernel,
+                                      int pool_type, int budget, void* out_k, void* out_v,
+                                      int32_t* out_idx, void* workspace, size_t workspace_bytes,
+                                      void* stream) {
+  snapkv_status_t st = check_common(B, Hq, Hkv, L, d, W);
+  if (st != SNAPKV_OK) return st;
+  st = check_pool(pool_kernel, pool_type);
+  if (st != SNAPKV_OK) return st;
+  if (budget <= W || !q_obs || !k_pool || !v_pool || !out_k || !out_v || !page_table)
+    return SNAPKV_ERR_INVALID_ARG;
+  if (!aligned16(q_obs) || !aligned16(k_pool) || !aligned16(v_pool) || !aligned16(out_k) ||
+      !aligned16(out_v) || (reinterpret_cast<uintptr_t>(page_table) & 3))
+    return SNAPKV_ERR_INVALID_ARG;
+  if (lse_obs && (reinterpret_cast<uintptr_t>(lse_obs) & 3)) return SNAPKV_ERR_INVALID_ARG;
+  // a tile of TILE_KEYS keys must lie inside one page
+  if (page_size < TILE_KEYS || page_size % TILE_KEYS != 0 || num_pages < 1 || pages_per_seq < 1)
+    return SNAPKV_ERR_INVALID_ARG;
+  if (static_cast<long long>(pages_per_seq) * page_size < L) return SNAPKV_ERR_INVALID_ARG;
+  KVStrides ks, vs;
+  if (!strides_ok(k_strides, d, &ks) || !strides_ok(v_strides, d, &vs)) return SNAPKV_ERR_INVALID_ARG;
+  const PagedKV paged_all = {page_table, pages_per_seq, page_size, num_pages};
+  if (!seq_lens)
+    return compress_impl(q_obs, k_pool, v_pool, B, Hq, Hkv, L, d, W, pool_kernel, pool_type, budget,
+                         out_k, out_v, out_idx, workspace, workspace_bytes, stream, false, lse_obs,
+                         &ks, &vs, false, &paged_all);
+  // per-sequence lengths: one single-sequence step each, as in snapkv_compress_varlen; every
+  // sequence and the workspace are checked before the first launch
+  for (int b = 0; b < B; ++b) {
+    if (seq_lens[b] < W || seq_lens[b] > L) return SNAPKV_ERR_INVALID_ARG;
+    if (!out_idx && seq_lens[b] > W) return SNAPKV_ERR_INVALID_ARG;
+  }
+  for (int b = 0; b < B; ++b) {
+    if (budget >= seq_lens[b]) continue;
+    const size_t need =
+        snapkv_workspace_size(1, Hq, Hkv, seq_lens[b], d, W, pool_kernel, pool_type, budget);
+    if (need == 0) return SNAPKV_ERR_INVALID_ARG;
+    if (!workspace_ok(workspace, workspace_bytes, need)) return SNAPKV_ERR_WORKSPACE;
+  }
+  if (workspace_ok(workspace, workspace_bytes, STATUS_BYTES) &&
+      clear_status(workspace, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return SNAPKV_ERR_CUDA;
+  const size_t head_rows = static_cast<size_t>(Hq) * budget * d * 2;
+  int launches = 0;
+  for (int b = 0; b < B; ++b) {
+    const PagedKV one = {page_table + static_cast<size_t>(b) * pages_per_seq, pages_per_seq,
+                         page_size, num_pages};
+    st = compress_impl(static_cast<const uint8_t*>(q_obs) + static_cast<size_t>(b) * Hq * W * d * 2,
+                       k_pool, v_pool, 1, Hq, Hkv, seq_lens[b], d, W, pool_kernel, pool_type, budget,
+                       static_cast<uint8_t*>(out_k) + b * head_rows,
+                       static_cast<uint8_t*>(out_v) + b * head_rows,
+                       out_idx ? out_idx + static_cast<size_t>(b) * Hq * (budget - W) : nullptr,
+                       workspace, workspace_bytes, stream, /*keep_status=*/true,
+                       lse_obs ? lse_obs + static_cast<size_t>(b) * Hq * W : nullptr, &ks, &vs, false,
+                       &one);
     if (st != SNAPKV_OK) return st;
     launches += g_last_launches;
   }

@@ -32,19 +32,25 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
                : "memory");
 }
 
-// Strides of K and of V in 16-byte vectors (batch, KV head, position).
+// Strides of K and of V in 16-byte vectors (batch or page, KV head, position).
 struct GatherStrides {
   long long kb, kh, kl, vb, vh, vl;
+};
+
+// Block table of a paged cache (table == nullptr: dense addressing).
+struct GatherPages {
+  const int32_t* table;
+  int pages_per_seq, page_size, num_pages;
 };
 
 // VPR = 16-byte vectors per row.  blockIdx.y (+ h0) is the (batch, query head) pair, blockIdx.x
 // a block of RPB consecutive output rows of that head; one thread moves one vector of K and
 // of V for GATHER_UNROLL rows, all loads issued before the first store.
-template <int VPR>
+template <int VPR, bool PAGED>
 __global__ void __launch_bounds__(GATHER_THREADS, GATHER_MIN_BLOCKS)
 gather_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v, const GatherStrides st,
-              const int32_t* __restrict__ idx, int h0, int g, int Hkv, int L, int W, int ksel,
-              int out_stride, uint4* __restrict__ out_k, uint4* __restrict__ out_v) {
+              const GatherPages pg, const int32_t* __restrict__ idx, int h0, int g, int Hkv, int L,
+              int W, int ksel, int out_stride, uint4* __restrict__ out_k, uint4* __restrict__ out_v) {
   constexpr int RPT = GATHER_THREADS / VPR;      // rows covered by the block per unrolled step
   constexpr int RPB = RPT * GATHER_UNROLL;       // rows per block
   const int rows = ksel + W;
@@ -54,8 +60,10 @@ gather_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v, const Ga
   const int t0 = blockIdx.x * RPB + threadIdx.x / VPR;
   const int kvh = bh / g;
   const int b = kvh / Hkv, c = kvh - b * Hkv;
-  const uint4* k_head = k + (b * st.kb + c * st.kh + vec);
-  const uint4* v_head = v + (b * st.vb + c * st.vh + vec);
+  // dense: the head's first row; paged: the head's first row inside page 0 of the pool
+  const uint4* k_head = k + ((PAGED ? 0 : b * st.kb) + c * st.kh + vec);
+  const uint4* v_head = v + ((PAGED ? 0 : b * st.vb) + c * st.vh + vec);
+  const int32_t* pages = PAGED ? pg.table + static_cast<size_t>(b) * pg.pages_per_seq : nullptr;
   const size_t dst_head = static_cast<size_t>(bh) * out_stride * VPR + vec;
   const int32_t* idx_head = idx ? idx + static_cast<size_t>(bh) * ksel : nullptr;
   int pos[GATHER_UNROLL];
@@ -71,8 +79,21 @@ gather_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v, const Ga
 #pragma unroll
   for (int uu = 0; uu < GATHER_UNROLL; ++uu)
     if (ok[uu]) {
-      kk[uu] = ld_stream(k_head + pos[uu] * st.kl);
-      vv[uu] = ld_stream(v_head + pos[uu] * st.vl);
+      if (PAGED) {
+        const int slot = pos[uu] / pg.page_size;
+        const int row = pos[uu] - slot * pg.page_size;
+        const int page = __ldg(pages + slot);
+        if (static_cast<unsigned>(page) < static_cast<unsigned>(pg.num_pages)) {
+          kk[uu] = ld_stream(k_head + page * st.kb + row * st.kl);
+          vv[uu] = ld_stream(v_head + page * st.vb + row * st.vl);
+        } else {  // an entry that names no page of the pool: zeros, as the scoring pass reads it
+          kk[uu] = make_uint4(0u, 0u, 0u, 0u);
+          vv[uu] = make_uint4(0u, 0u, 0u, 0u);
+        }
+      } else {
+        kk[uu] = ld_stream(k_head + pos[uu] * st.kl);
+        vv[uu] = ld_stream(v_head + pos[uu] * st.vl);
+      }
     }
 #pragma unroll
   for (int uu = 0; uu < GATHER_UNROLL; ++uu)
@@ -88,7 +109,7 @@ gather_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v, const Ga
 cudaError_t launch_gather(const void* k, const void* v, const KVStrides& ks, const KVStrides& vs,
                           const int32_t* idx, int B, int Hq, int Hkv, int L, int d, int W, int ksel,
                           int out_rows_stride, void* out_k, void* out_v, cudaStream_t stream,
-                          int* launches) {
+                          int* launches, const PagedKV* paged) {
   const int rows = ksel + W;
   const int vpr = d * 2 / 16;
   const int rpb = GATHER_THREADS / vpr * GATHER_UNROLL;
@@ -107,12 +128,24 @@ cudaError_t launch_gather(const void* k, const void* v, const KVStrides& ks, con
   for (long long h0 = 0; h0 < heads; h0 += slab) {
     const unsigned gy = static_cast<unsigned>(heads - h0 < slab ? heads - h0 : slab);
     const int h0i = static_cast<int>(h0);
-    if (vpr == 16)
-      gather_kernel<16><<<dim3(gx, gy), GATHER_THREADS, 0, stream>>>(
-          kp, vp, st, idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
-    else
-      gather_kernel<8><<<dim3(gx, gy), GATHER_THREADS, 0, stream>>>(
-          kp, vp, st, idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
+    const dim3 grid(gx, gy);
+    if (paged) {
+      const GatherPages pg = {paged->table, paged->pages_per_seq, paged->page_size, paged->num_pages};
+      if (vpr == 16)
+        gather_kernel<16, true><<<grid, GATHER_THREADS, 0, stream>>>(
+            kp, vp, st, pg, idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
+      else
+        gather_kernel<8, true><<<grid, GATHER_THREADS, 0, stream>>>(
+            kp, vp, st, pg, idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
+    } else {
+      const GatherPages pg = {nullptr, 0, 1, 0};
+      if (vpr == 16)
+        gather_kernel<16, false><<<grid, GATHER_THREADS, 0, stream>>>(
+            kp, vp, st, pg, idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
+      else
+        gather_kernel<8, false><<<grid, GATHER_THREADS, 0, stream>>>(
+            kp, vp, st, pg, idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
+    }
     *launches += 1;
   }
   return cudaGetLastError();

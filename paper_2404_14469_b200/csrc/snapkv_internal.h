@@ -82,6 +82,17 @@ class DeviceOnce {
   std::atomic<bool> flags_[MAX_DEV] = {};
 };
 
+// Block-table addressing of K and V (a serving stack's paged cache): position p of sequence b
+// is row p % page_size of page table[b * pages_per_seq + p / page_size] of a pool of pages.
+// With a table, a KVStrides' `b` is the element stride between consecutive PAGES of the pool,
+// `h` between KV heads inside a page and `l` between positions inside a page.
+struct PagedKV {
+  const int32_t* table;  // device memory; nullptr = not paged
+  int pages_per_seq;     // entries per sequence (row stride of the table)
+  int page_size;         // positions per page, a multiple of TILE_KEYS
+  int num_pages;         // pages in the pool; an entry outside [0, num_pages) reads as zeros
+};
+
 struct WorkspaceLayout {
   size_t off_status, off_counters, off_partials, off_lse, off_vote, off_pooled, total;
 };
@@ -115,7 +126,8 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrid
                                  float* vote, int* status,
                                  int* counters, float* partials, float* lse2, cudaStream_t stream,
                                  int* launches, const float* lse_obs = nullptr,
-                                 bool keep_status = false, bool never_ready = false);
+                                 bool keep_status = false, bool never_ready = false,
+                                 const PagedKV* paged = nullptr);
 
 // Pool + top-k over `rows` rows of fp32 votes.  `pooled_scratch` (select_scratch_bytes bytes)
 // is only touched when select_needs_scratch(n).  With gsum > 1 a selection row is the sum of
@@ -125,11 +137,18 @@ cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel
                              int ksel, int32_t* out_idx, float* pooled_scratch,
                              cudaStream_t stream, int* launches, int gsum = 1);
 
+// The one-cluster-per-row select kernel: whether it takes rows of this length and pooling
+// kernel on the current device, and its launch (same contract as launch_pool_topk, no scratch).
+bool select_cluster_applies(int rows, int n, int pool_kernel);
+cudaError_t launch_pool_topk_cluster(const float* vote, int rows, int n, int pool_kernel,
+                                     int pool_type, int ksel, int32_t* out_idx, cudaStream_t stream,
+                                     int* launches, int gsum);
+
 // Gather + append.  idx == nullptr copies rows 0..ksel-1 (identity path).
 cudaError_t launch_gather(const void* k, const void* v, const KVStrides& ks, const KVStrides& vs,
                           const int32_t* idx, int B, int Hq, int Hkv, int L, int d, int W, int ksel,
                           int out_rows_stride, void* out_k, void* out_v, cudaStream_t stream,
-                          int* launches);
+                          int* launches, const PagedKV* paged = nullptr);
 
 cudaError_t launch_iota_idx(int32_t* out_idx, int rows, int n, int row_stride, cudaStream_t stream,
                             int* launches);

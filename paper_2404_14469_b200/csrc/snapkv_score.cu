@@ -75,6 +75,8 @@ struct ScoreArgs {
   int pipelined;            // how many waves the statistics run ahead of the votes (>= 1)
   int votes_only;           // 1: lse2 and the counters are already set, no statistics pass
   unsigned long long wait_ns;  // time limit of every device-side wait
+  const int32_t* page_table;   // paged K: [batch][pages_per_seq] page numbers, else nullptr
+  int pages_per_seq, page_size;
   float c2;                 // log2(e) / sqrt(d)
   float* partials;          // [units][maxseg][MAX_COLS] log2-sum-exp of one CTA's share
   float* lse2;              // [units][MAX_COLS] minus the log2-sum-exp per window row, when supplied
@@ -323,14 +325,21 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           const uint32_t ph = (git / STAGES) & 1;
           if (!mbar_wait_thread(bar_empty(s), ph ^ 1, abort_s, WAIT_PRODUCER_EMPTY)) return false;
           mbar_expect_tx(bar_full(s), SM::STAGE_BYTES);
-          const int key0 = tile_of(it, k) * TILE_KEYS;
+          int key0 = tile_of(it, k) * TILE_KEYS;
+          int kslab = kb;  // outermost coordinate of the K map: the batch, or the page of the pool
+          if (a.page_table) {
+            // a page holds a whole number of tiles: the tile's 128 keys sit in one page
+            const int pg = key0 / a.page_size;
+            kslab = __ldg(a.page_table + static_cast<size_t>(kb) * a.pages_per_seq + pg);
+            key0 -= pg * a.page_size;
+          }
           // the vote pass is the last reader of a key tile: its lines may leave L2 first,
           // which keeps the next wave's statistics-pass lines resident instead
           for (int sb = 0; sb < SUBT; ++sb) {
             if (it.vote)
-              tma_load_4d_hint(stage_addr(s, sb), &tmK, bar_full(s), sb * 64, key0, kh, kb, pol_first);
+              tma_load_4d_hint(stage_addr(s, sb), &tmK, bar_full(s), sb * 64, key0, kh, kslab, pol_first);
             else
-              tma_load_4d(stage_addr(s, sb), &tmK, bar_full(s), sb * 64, key0, kh, kb);
+              tma_load_4d(stage_addr(s, sb), &tmK, bar_full(s), sb * 64, key0, kh, kslab);
           }
         }
         return true;
@@ -927,13 +936,17 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrid
                                  float* vote, int* status,
                                  int* counters, float* partials, float* lse2, cudaStream_t stream,
                                  int* launches, const float* lse_obs, bool keep_status,
-                                 bool never_ready) {
+                                 bool never_ready, const PagedKV* paged) {
   CUtensorMap tmK, tmQ;
   {
     // (d, position, KV head, batch) with the caller's strides: any layout whose rows of d
-    // elements are contiguous is one tensor map, e.g. [B, L, Hkv, d] as well as [B, Hkv, L, d]
-    cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(L),
-                          static_cast<cuuint64_t>(Hkv), static_cast<cuuint64_t>(B)};
+    // elements are contiguous is one tensor map, e.g. [B, L, Hkv, d] as well as [B, Hkv, L, d].
+    // A paged cache is the same map over the pool: (d, position in page, KV head, page); rows
+    // past a page's end or pages outside the pool read as zeros.
+    cuuint64_t dims[4] = {static_cast<cuuint64_t>(d),
+                          static_cast<cuuint64_t>(paged ? paged->page_size : L),
+                          static_cast<cuuint64_t>(Hkv),
+                          static_cast<cuuint64_t>(paged ? paged->num_pages : B)};
     cuuint64_t strides[3] = {static_cast<cuuint64_t>(ks.l) * 2, static_cast<cuuint64_t>(ks.h) * 2,
                              static_cast<cuuint64_t>(ks.b) * 2};
     cuuint32_t box[4] = {64, TILE_KEYS, 1, 1};
@@ -947,6 +960,9 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrid
   }
   ScoreArgs a = schedule_args(plan, L, W, Hkv, (lse_obs || never_ready) ? 1 : 0);
   a.wait_ns = wait_limit_setting();
+  a.page_table = paged ? paged->table : nullptr;
+  a.pages_per_seq = paged ? paged->pages_per_seq : 0;
+  a.page_size = paged ? paged->page_size : 1;
   a.c2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
   a.partials = partials;
   a.lse2 = lse2;

@@ -777,7 +777,16 @@ cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel
     once.set();
   }
   const int r = pool_kernel >> 1;
-  if (n <= FAST_MAX_KEYS && r <= 7) {
+  // One cluster of small CTAs per row: for rows too long for the one-CTA kernel below, and
+  // whenever there are too few rows to fill the GPU with one CTA each.  The cluster kernel's
+  // chain of cluster barriers takes about 17-21 us whatever the row count (measured: 32 rows
+  // of 32736 in 21 us, 64 in 25 us, 128 in 45 us); the one-CTA kernel takes about 26-28 us for
+  // any number of rows up to the SM count.
+  const bool one_cta_fits = n <= FAST_MAX_KEYS && r <= 7;
+  if ((!one_cta_fits || rows <= 48) && select_cluster_applies(rows, n, pool_kernel))
+    return launch_pool_topk_cluster(vote, rows, n, pool_kernel, pool_type, ksel, out_idx, stream,
+                                    launches, gsum);
+  if (one_cta_fits) {
     const int ept = (((n + SEL_THREADS - 1) / SEL_THREADS) + 7) & ~7;
     const int words = key_slot4_host(SEL_THREADS * ept) + 4;
 #define SNAPKV_FAST_LAUNCH(RM, P)                                                            \

@@ -107,6 +107,25 @@ def test_uniform_attention_closed_form_on_gpu():
     (1, 49152, 13, "max", 8128),
     (3, 32736, 13, "avg", 4064),    # radius 6 with its own instantiation
     (2, 16352, 3, "max", 992),      # radius 1: run-time radius path
+    # one cluster of CTAs per row: 4096 to 131072 positions, pooling radius up to 7
+    (3, 4095, 7, "max", 500),       # just below: one CTA per row
+    (3, 4096, 7, "max", 500),       # two CTAs of 8 keys a thread
+    (2, 4100, 5, "avg", 4099),
+    (2, 16384, 15, "avg", 2016),    # radius 7, run-time radius
+    (2, 16385, 7, "max", 2016),     # 16 keys a thread, last CTA nearly empty
+    (4, 32736, 5, "avg", 4064),     # the 32K workload's rows: 8 CTAs of 16 keys a thread
+    (2, 65536, 7, "max", 8128),     # 8 CTAs of 32 keys a thread, full
+    (2, 65537, 7, "max", 8128),     # 16 CTAs
+    (2, 131008, 7, "max", 8128),    # the 128K workload's rows
+    (1, 131072, 5, "avg", 2016),
+    (1, 131073, 7, "max", 2016),    # one more: many-CTA path with global scratch
+    (2, 140000, 7, "max", 4064),
+    (1, 150001, 5, "avg", 1000),
+    (50, 20000, 7, "max", 2016),    # more rows than the cluster kernel takes on: one CTA per row
+    (49, 32736, 5, "avg", 4064),
+    (64, 40960, 13, "max", 31000),
+    (2, 20000, 17, "max", 2016),    # radius 8: beyond the cluster kernel, one CTA per row
+    (1, 70000, 17, "avg", 2016),    # radius 8, long row: many-CTA path
 ])
 def test_pool_topk_matches_oracle(rows, n, kernel, ptype, ksel):
     g = torch.Generator().manual_seed(n + kernel)
@@ -156,13 +175,15 @@ def test_compress_that_keeps_all_but_one_row_of_a_long_prompt():
     _check_compress(data, W, 5, "avg", budget)
 
 
-def test_pool_topk_exact_ties_take_lower_positions():
-    n, ksel = 5000, 700
-    vote = torch.zeros(2, n)
+@pytest.mark.parametrize("n,ksel", [(3000, 700), (5000, 700), (40000, 9000), (100000, 30000), (200000, 1234)])
+def test_pool_topk_exact_ties_take_lower_positions(n, ksel):
+    vote = torch.zeros(3, n)
     vote[0, :] = 0.25                         # all equal: the first ksel positions win
     vote[1, 100::10] = 1.0                    # plateaus of width 7 around every tenth position
+    vote[2, :] = 0.0                          # all zero: again the first ksel positions
     idx = sk.snapkv_pool_topk(vote.cuda(), 7, sk.POOL_MAX, ksel).cpu().numpy()
     assert np.array_equal(idx[0], np.arange(ksel))
+    assert np.array_equal(idx[2], np.arange(ksel))
     pooled = orc.pool1d(vote[1].numpy().astype(np.float64), 7, orc.POOL_MAX)
     assert np.array_equal(idx[1], orc.topk_positions(pooled, ksel))
 
