@@ -368,6 +368,50 @@ snapkv_status_t snapkv_compress_paged(const void* q_obs, const void* k_pool, con
                                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * A prompt sharded along its length (context parallelism).  The paper stops at what one GPU
+ * holds (Sec. 5.1.1: 380K tokens; Sec. 6 leaves prompt processing aside); Eq. 1-2 decompose
+ * over ranges of keys, which is what these four per-shard steps implement.  A shard holds
+ * the keys and values of positions [pos0, pos0 + Ls) of every sequence, dense
+ * [B, Hkv, Ls, d], and all shards know q_obs (the last W queries of the whole prompt).  With
+ * n = L_total - W the whole prompt's prefix length:
+ *
+ * 1. snapkv_shard_lse: the shard's share of each window row's softmax normaliser.
+ *    out_lse fp32 [B, Hq, W] = log sum over the shard's keys j visible to window row i
+ *    (global position pos0 + j <= n + i, i.e. local j <= mask_n + i with mask_n = n - pos0,
+ *    which may be negative or exceed Ls) of exp(q_i.k_j / sqrt(d)); -inf where a row sees no
+ *    key of the shard.  Requires W <= Ls.
+ * 2. snapkv_lse_merge: out[i] = log sum_r exp(parts[r][i]) over R shards' results laid out
+ *    [R][count] (count = B*Hq*W), folded in the order of r, so every rank that merges the same
+ *    gathered buffer gets the same bits.  This is lse_obs of snapkv_window_scores_lse.
+ * 3. snapkv_shard_votes: Eq. 1 for the shard's first n_vote keys (those of its keys that are
+ *    prefix keys: min(Ls, n - pos0)) given the merged lse_obs:
+ *    out_vote fp32 [B, Hq, n_vote].  Concatenated over the shards these are the votes of the
+ *    whole prompt; pooling and top-k then run on the whole rows (snapkv_pool_topk).
+ * 4. snapkv_gather_range: the shard's part of the gather.  idx int32 [B, Hq, ksel] holds a
+ *    head's selected GLOBAL positions, ascending; the entries inside [pos0, pos0 + Ls) form
+ *    one segment.  Their K/V rows are copied to rows [0, count) of out_k/out_v
+ *    [B, Hq, out_rows, d], followed by the shard's last `append` rows (the window rows, on
+ *    the shard that holds them; 0 elsewhere); seg int32 [B, Hq, 2] = {first entry of the
+ *    segment, count}.  out_rows >= min(ksel, Ls) + append.  The whole compressed cache of a
+ *    head is the shards' segments in shard order, then the window rows.
+ * Workspaces: snapkv_workspace_size(B, Hq, Hkv, Ls, d, W, 1, 0, W + 1) bytes suffice for
+ * steps 1 and 3.  Everything else as for the single-GPU entry points.
+ */
+snapkv_status_t snapkv_shard_lse(const void* q_obs, const void* k_shard,
+                                 int B, int Hq, int Hkv, int Ls, int d, int W, int mask_n,
+                                 float* out_lse,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+snapkv_status_t snapkv_lse_merge(const float* parts, int R, int count, float* out, void* stream);
+snapkv_status_t snapkv_shard_votes(const void* q_obs, const void* k_shard, const float* lse_obs,
+                                   int B, int Hq, int Hkv, int Ls, int d, int W, int n_vote,
+                                   float* out_vote,
+                                   void* workspace, size_t workspace_bytes, void* stream);
+snapkv_status_t snapkv_gather_range(const void* k_shard, const void* v_shard, const int32_t* idx,
+                                    int B, int Hq, int Hkv, int Ls, int d, int pos0, int ksel,
+                                    int append, void* out_k, void* out_v, int out_rows,
+                                    int32_t* seg, void* stream);
+
+/*
  * The scoring kernel's schedule, for inspection (no counterpart in the paper).  The kernel
  * is a persistent grid; every block walks a fixed list of work items - tiles [t0, t1) of 128
  * keys of one unit (a batch, a KV head and up to 128 window columns of its query heads), in

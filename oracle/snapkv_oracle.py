@@ -41,6 +41,10 @@ sequence b is row p % page_size of page table[b][p // page_size] of a pool), one
 at a time, and then run the very same step: paging changes where a row lives, not what the
 method computes.
 
+shard_lse / merge_lse / shard_votes split Eq. 1 over ranges of keys (a prompt sharded along
+its length): a row's normaliser is the sum of the shards' shares, and a key's vote needs only
+its own logits and the merged normalisers.
+
 hit_counts / hit_rate state the paper's hit-rate measure of a selection (Sec. 3, Eq. 3-7);
 decode_attention is the generation step's attention over the compressed cache (Sec. 5.1.2).
 
@@ -356,6 +360,38 @@ def compress_grouped(q_obs: np.ndarray, k: np.ndarray, v: np.ndarray, pool_kerne
             out_k[b, c, ksel:] = k[b, c, n:]
             out_v[b, c, ksel:] = v[b, c, n:]
     return {"out_k": out_k, "out_v": out_v, "out_idx": out_idx, "vote": vote, "pooled": pooled}
+
+
+def shard_lse(q_head: np.ndarray, k_shard_head: np.ndarray, pos0: int, n_total: int) -> np.ndarray:
+    """One head, one shard holding positions [pos0, pos0 + Ls) of the prompt: for every window
+    row i the log of the sum of exp(logit) over the shard's keys the row may see (global
+    position <= n_total + i).  -inf where the row sees none of them.  [W] fp64."""
+    W = q_head.shape[0]
+    Ls = k_shard_head.shape[0]
+    s = window_logits(q_head, k_shard_head)          # [W, Ls]
+    out = np.full(W, -np.inf)
+    for i in range(W):
+        seen = min(Ls, n_total + i - pos0 + 1)       # local keys 0 .. seen-1
+        if seen > 0:
+            row = s[i, :seen]
+            m = row.max()
+            out[i] = m + math.log(np.exp(row - m).sum())
+    return out
+
+
+def merge_lse(parts: np.ndarray) -> np.ndarray:
+    """log sum_r exp(parts[r]) over the first axis (the shards' shares of a normaliser)."""
+    m = parts.max(axis=0)
+    safe = np.where(np.isfinite(m), m, 0.0)
+    return safe + np.log(np.exp(parts - safe).sum(axis=0))
+
+
+def shard_votes(q_head: np.ndarray, k_shard_head: np.ndarray, lse: np.ndarray, n_vote: int) -> np.ndarray:
+    """Eq. 1 for the first n_vote keys of a shard, given every window row's log-sum-exp over
+    the WHOLE prompt: vote_j = sum_i exp(logit_ij - lse_i).  Prefix keys are seen by every row,
+    so no mask is involved.  [n_vote] fp64."""
+    s = window_logits(q_head, k_shard_head[:n_vote])
+    return np.exp(s - lse[:, None]).sum(axis=0)
 
 
 def read_paged(pool: np.ndarray, table_row, page_size: int, length: int) -> np.ndarray:

@@ -30,6 +30,7 @@ SYMBOLS = [
     "snapkv_hit_counts", "snapkv_decode_workspace_size", "snapkv_decode_attention",
     "snapkv_set_wait_limit_ns", "snapkv_selftest_stalled_scores", "snapkv_schedule_items",
     "snapkv_compress_paged",
+    "snapkv_shard_lse", "snapkv_lse_merge", "snapkv_shard_votes", "snapkv_gather_range",
 ]
 
 _lib = None
@@ -76,6 +77,14 @@ def lib() -> ctypes.CDLL:
     L.snapkv_compress_paged.restype = c_int
     L.snapkv_compress_paged.argtypes = ([c_vp] * 3 + [p64] * 2 + [c_vp] + [c_int] * 3 + [p32, c_vp]
                                         + [c_int] * 9 + [c_vp] * 3 + [c_vp, c_sz, c_vp])
+    L.snapkv_shard_lse.restype = c_int
+    L.snapkv_shard_lse.argtypes = [c_vp] * 2 + [c_int] * 7 + [c_vp, c_vp, c_sz, c_vp]
+    L.snapkv_lse_merge.restype = c_int
+    L.snapkv_lse_merge.argtypes = [c_vp, c_int, c_int, c_vp, c_vp]
+    L.snapkv_shard_votes.restype = c_int
+    L.snapkv_shard_votes.argtypes = [c_vp] * 3 + [c_int] * 7 + [c_vp, c_vp, c_sz, c_vp]
+    L.snapkv_gather_range.restype = c_int
+    L.snapkv_gather_range.argtypes = [c_vp] * 3 + [c_int] * 8 + [c_vp, c_vp, c_int, c_vp, c_vp]
     L.snapkv_hit_counts.restype = c_int
     L.snapkv_hit_counts.argtypes = [c_vp, c_vp, c_int, c_int, c_int, ctypes.c_float, c_vp, c_vp]
     L.snapkv_decode_workspace_size.restype = c_sz
@@ -317,6 +326,66 @@ def snapkv_compress_paged(q_obs, k_pool, v_pool, page_table, L, pool_kernel: int
         workspace.data_ptr(), workspace.numel(), _stream_ptr())
     _check(code, "snapkv_compress_paged")
     return out_k, out_v, out_idx, workspace
+
+
+def snapkv_shard_lse(q_obs, k_shard, mask_n: int, workspace=None):
+    """A shard's partial log-sum-exp of every window row: fp32 [B, Hq, W] (and the workspace)."""
+    _dev_bf16(q_obs, "q_obs"), _dev_bf16(k_shard, "k_shard")
+    B, Hq, Hkv, Ls, d, W = _shapes(q_obs, k_shard)
+    L_ = lib()
+    need = L_.snapkv_workspace_size(B, Hq, Hkv, Ls, d, W, 1, 0, W + 1)
+    if workspace is None or workspace.numel() < need:
+        workspace = _alloc_ws(need, k_shard.device)
+    out = torch.empty(B, Hq, W, dtype=torch.float32, device=k_shard.device)
+    code = L_.snapkv_shard_lse(q_obs.data_ptr(), k_shard.data_ptr(), B, Hq, Hkv, Ls, d, W, int(mask_n),
+                               out.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream_ptr())
+    _check(code, "snapkv_shard_lse")
+    return out, workspace
+
+
+def snapkv_lse_merge(parts):
+    """parts fp32 [R, ...] (CUDA, contiguous) -> log-sum-exp over the first axis, in its order."""
+    if not (parts.is_cuda and parts.dtype == torch.float32 and parts.is_contiguous() and parts.dim() >= 2):
+        raise SnapKVError("parts must be a contiguous CUDA fp32 [R, ...] tensor")
+    out = torch.empty(parts.shape[1:], dtype=torch.float32, device=parts.device)
+    code = lib().snapkv_lse_merge(parts.data_ptr(), parts.shape[0], out.numel(), out.data_ptr(), _stream_ptr())
+    _check(code, "snapkv_lse_merge")
+    return out
+
+
+def snapkv_shard_votes(q_obs, k_shard, lse_obs, n_vote: int, workspace=None):
+    """Votes of a shard's first n_vote keys given the merged normalisers: fp32 [B, Hq, n_vote]."""
+    _dev_bf16(q_obs, "q_obs"), _dev_bf16(k_shard, "k_shard")
+    B, Hq, Hkv, Ls, d, W = _shapes(q_obs, k_shard)
+    L_ = lib()
+    need = L_.snapkv_workspace_size(B, Hq, Hkv, Ls, d, W, 1, 0, W + 1)
+    if workspace is None or workspace.numel() < need:
+        workspace = _alloc_ws(need, k_shard.device)
+    out = torch.empty(B, Hq, n_vote, dtype=torch.float32, device=k_shard.device)
+    code = L_.snapkv_shard_votes(q_obs.data_ptr(), k_shard.data_ptr(), _lse_arg(lse_obs, B, Hq, W), B, Hq, Hkv,
+                                 Ls, d, W, int(n_vote), out.data_ptr(), workspace.data_ptr(),
+                                 workspace.numel(), _stream_ptr())
+    _check(code, "snapkv_shard_votes")
+    return out, workspace
+
+
+def snapkv_gather_range(k_shard, v_shard, idx, pos0: int, append: int):
+    """The shard's segment of every head's selected rows (+ `append` trailing rows of the shard).
+    Returns (out_k, out_v [B, Hq, min(ksel, Ls) + append, d], seg int32 [B, Hq, 2])."""
+    _dev_bf16(k_shard, "k_shard"), _dev_bf16(v_shard, "v_shard")
+    if not (idx.is_cuda and idx.dtype == torch.int32 and idx.is_contiguous() and idx.dim() == 3):
+        raise SnapKVError("idx must be a contiguous CUDA int32 [B, Hq, ksel] tensor")
+    B, Hkv, Ls, d = k_shard.shape
+    _, Hq, ksel = idx.shape
+    rows = min(ksel, Ls) + append
+    out_k = torch.zeros(B, Hq, rows, d, dtype=torch.bfloat16, device=k_shard.device)
+    out_v = torch.zeros_like(out_k)
+    seg = torch.empty(B, Hq, 2, dtype=torch.int32, device=k_shard.device)
+    code = lib().snapkv_gather_range(k_shard.data_ptr(), v_shard.data_ptr(), idx.data_ptr(), B, Hq, Hkv, Ls, d,
+                                     int(pos0), ksel, int(append), out_k.data_ptr(), out_v.data_ptr(), rows,
+                                     seg.data_ptr(), _stream_ptr())
+    _check(code, "snapkv_gather_range")
+    return out_k, out_v, seg
 
 
 def snapkv_hit_counts(a_cur, idx, theta: float):

@@ -122,6 +122,20 @@ static snapkv_status_t check_pool(int pool_kernel, int pool_type) {
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// out[i] = log sum_r exp(parts[r][i]), folded in the order of r (the same on every rank).
+__global__ void lse_merge_kernel(const float* __restrict__ parts, int R, int count, float* __restrict__ out) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  float M = -INFINITY, S = 0.f;
+  for (int r = 0; r < R; ++r) {
+    const float p = parts[static_cast<size_t>(r) * count + i];
+    const float Mn = fmaxf(fmaxf(M, p), -1e30f);
+    S = S * expf(M - Mn) + expf(p - Mn);
+    M = Mn;
+  }
+  out[i] = M + logf(S);
+}
+
 }  // namespace snapkv
 
 using namespace snapkv;
@@ -496,6 +510,97 @@ snapkv_status_t snapkv_compress_paged(const void* q_obs, const void* k_pool, con
   }
   g_last_launches = launches;
   return SNAPKV_OK;
+}
+
+// ---- a prompt sharded along its length over several GPUs: the per-shard steps
+static snapkv_status_t shard_common(const void* q_obs, const void* k_shard, int B, int Hq, int Hkv,
+                                    int Ls, int d, int W) {
+  snapkv_status_t st = check_common(B, Hq, Hkv, Ls, d, W);
+  if (st != SNAPKV_OK) return st;
+  if (!q_obs || !k_shard || !aligned16(q_obs) || !aligned16(k_shard)) return SNAPKV_ERR_INVALID_ARG;
+  return SNAPKV_OK;
+}
+
+snapkv_status_t snapkv_shard_lse(const void* q_obs, const void* k_shard, int B, int Hq, int Hkv,
+                                 int Ls, int d, int W, int mask_n, float* out_lse, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
+  snapkv_status_t st = shard_common(q_obs, k_shard, B, Hq, Hkv, Ls, d, W);
+  if (st != SNAPKV_OK) return st;
+  if (!out_lse || (reinterpret_cast<uintptr_t>(out_lse) & 3)) return SNAPKV_ERR_INVALID_ARG;
+  ScorePlan p;
+  if (!make_score_plan(B, Hq, Hkv, Ls, d, W, &p)) return SNAPKV_ERR_UNSUPPORTED;
+  const WorkspaceLayout w = make_layout(p, B, Hq, 0, false, false);
+  if (!workspace_ok(workspace, workspace_bytes, w.total)) return SNAPKV_ERR_WORKSPACE;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (launch_clear(ws, w, s) != cudaSuccess) return SNAPKV_ERR_CUDA;
+  int launches = 1;
+  const ShardMode shard = {mask_n, out_lse};
+  if (launch_window_scores(q_obs, k_shard, dense_strides(Hkv, Ls, d), B, Hq, Hkv, Ls, d, W, p, nullptr,
+                           reinterpret_cast<int*>(ws + w.off_status),
+                           reinterpret_cast<int*>(ws + w.off_counters),
+                           reinterpret_cast<float*>(ws + w.off_partials),
+                           reinterpret_cast<float*>(ws + w.off_lse), s, &launches, nullptr, false,
+                           false, nullptr, &shard) != cudaSuccess)
+    return SNAPKV_ERR_CUDA;
+  g_last_launches = launches;
+  return SNAPKV_OK;
+}
+
+snapkv_status_t snapkv_lse_merge(const float* parts, int R, int count, float* out, void* stream) {
+  if (!parts || !out || R < 1 || count < 1) return SNAPKV_ERR_INVALID_ARG;
+  lse_merge_kernel<<<(count + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(parts, R, count, out);
+  g_last_launches = 1;
+  return cudaGetLastError() == cudaSuccess ? SNAPKV_OK : SNAPKV_ERR_CUDA;
+}
+
+snapkv_status_t snapkv_shard_votes(const void* q_obs, const void* k_shard, const float* lse_obs,
+                                   int B, int Hq, int Hkv, int Ls, int d, int W, int n_vote,
+                                   float* out_vote, void* workspace, size_t workspace_bytes,
+                                   void* stream) {
+  snapkv_status_t st = shard_common(q_obs, k_shard, B, Hq, Hkv, Ls, d, W);
+  if (st != SNAPKV_OK) return st;
+  if (!lse_obs || !out_vote || n_vote < 1 || n_vote > Ls) return SNAPKV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(lse_obs) & 3) || (reinterpret_cast<uintptr_t>(out_vote) & 3))
+    return SNAPKV_ERR_INVALID_ARG;
+  ScorePlan p;
+  if (!make_score_plan(B, Hq, Hkv, Ls, d, W, &p, n_vote)) return SNAPKV_ERR_UNSUPPORTED;
+  const WorkspaceLayout w = make_layout(p, B, Hq, 0, false, false);
+  if (!workspace_ok(workspace, workspace_bytes, w.total)) return SNAPKV_ERR_WORKSPACE;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  int launches = 0;
+  if (launch_window_scores(q_obs, k_shard, dense_strides(Hkv, Ls, d), B, Hq, Hkv, Ls, d, W, p, out_vote,
+                           reinterpret_cast<int*>(ws + w.off_status),
+                           reinterpret_cast<int*>(ws + w.off_counters),
+                           reinterpret_cast<float*>(ws + w.off_partials),
+                           reinterpret_cast<float*>(ws + w.off_lse), static_cast<cudaStream_t>(stream),
+                           &launches, lse_obs) != cudaSuccess)
+    return SNAPKV_ERR_CUDA;
+  g_last_launches = launches;
+  return SNAPKV_OK;
+}
+
+snapkv_status_t snapkv_gather_range(const void* k_shard, const void* v_shard, const int32_t* idx,
+                                    int B, int Hq, int Hkv, int Ls, int d, int pos0, int ksel,
+                                    int append, void* out_k, void* out_v, int out_rows,
+                                    int32_t* seg, void* stream) {
+  if (B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || Ls < 1 || (d != 64 && d != 128))
+    return SNAPKV_ERR_INVALID_ARG;
+  if (pos0 < 0 || ksel < 0 || append < 0 || append > Ls || !k_shard || !v_shard || !out_k || !out_v || !seg ||
+      (ksel > 0 && !idx))
+    return SNAPKV_ERR_INVALID_ARG;
+  if (!aligned16(k_shard) || !aligned16(v_shard) || !aligned16(out_k) || !aligned16(out_v))
+    return SNAPKV_ERR_INVALID_ARG;
+  if (static_cast<long long>(B) * Hq > 65535) return SNAPKV_ERR_UNSUPPORTED;
+  const int most = (ksel < Ls ? ksel : Ls) + append;  // rows a head can get from this shard
+  if (out_rows < most) return SNAPKV_ERR_INVALID_ARG;
+  int launches = 0;
+  const KVStrides ds = dense_strides(Hkv, Ls, d);
+  const cudaError_t e = launch_gather_range(k_shard, v_shard, ds, ds, idx, B, Hq, Hkv, Ls, d, pos0, ksel,
+                                            append, out_rows, out_k, out_v, seg,
+                                            static_cast<cudaStream_t>(stream), &launches);
+  g_last_launches = launches;
+  return e == cudaSuccess ? SNAPKV_OK : SNAPKV_ERR_CUDA;
 }
 
 size_t snapkv_host_staging_size(int B, int Hq, int Hkv, int L, int d, int W, int pool_kernel,

@@ -104,7 +104,92 @@ gather_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v, const Ga
     }
 }
 
+// A shard of a longer prompt holds positions [pos0, pos0 + L).  Of a head's ascending list of
+// selected positions, the entries inside that range form one contiguous segment; this kernel
+// finds it (two binary searches per block) and copies those rows, then `append` trailing rows
+// of the shard (the window rows, on the shard that holds them), into rows [0, count + append)
+// of the head's output.  seg[head] = {first entry of the segment, entries in it}.
+template <int VPR>
+__global__ void __launch_bounds__(GATHER_THREADS, GATHER_MIN_BLOCKS)
+gather_range_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v, const GatherStrides st,
+                    const int32_t* __restrict__ idx, int g, int Hkv, int L, int pos0, int ksel, int append,
+                    int out_stride, uint4* __restrict__ out_k, uint4* __restrict__ out_v,
+                    int32_t* __restrict__ seg) {
+  constexpr int RPT = GATHER_THREADS / VPR;
+  constexpr int RPB = RPT * GATHER_UNROLL;
+  __shared__ int s_lo, s_cnt;
+  const int bh = blockIdx.y;
+  const int32_t* idx_head = idx + static_cast<size_t>(bh) * ksel;
+  if (threadIdx.x == 0) {
+    auto lower_bound = [&](int value) {  // first entry >= value
+      int lo = 0, hi = ksel;
+      while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(idx_head + mid) < value) lo = mid + 1; else hi = mid;
+      }
+      return lo;
+    };
+    const int lo = lower_bound(pos0);
+    const int hi = lower_bound(pos0 + L);
+    s_lo = lo;
+    s_cnt = hi - lo;
+    if (blockIdx.x == 0) {
+      seg[2 * bh] = lo;
+      seg[2 * bh + 1] = hi - lo;
+    }
+  }
+  __syncthreads();
+  const int lo = s_lo, cnt = s_cnt;
+  const int rows = cnt + append;
+  if (static_cast<int>(blockIdx.x) * RPB >= rows) return;
+  const int vec = threadIdx.x % VPR;
+  const int t0 = blockIdx.x * RPB + threadIdx.x / VPR;
+  const int kvh = bh / g;
+  const int b = kvh / Hkv, c = kvh - b * Hkv;
+  const uint4* k_head = k + (b * st.kb + c * st.kh + vec);
+  const uint4* v_head = v + (b * st.vb + c * st.vh + vec);
+  const size_t dst_head = static_cast<size_t>(bh) * out_stride * VPR + vec;
+#pragma unroll
+  for (int uu = 0; uu < GATHER_UNROLL; ++uu) {
+    const int t = t0 + uu * RPT;
+    if (t < rows) {
+      const int pos = t < cnt ? __ldg(idx_head + lo + t) - pos0 : L - append + (t - cnt);
+      const uint4 kk = ld_stream(k_head + pos * st.kl);
+      const uint4 vv = ld_stream(v_head + pos * st.vl);
+      const size_t dst = dst_head + static_cast<size_t>(t) * VPR;
+      st_stream(out_k + dst, kk);
+      st_stream(out_v + dst, vv);
+    }
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_gather_range(const void* k, const void* v, const KVStrides& ks, const KVStrides& vs,
+                                const int32_t* idx, int B, int Hq, int Hkv, int L, int d, int pos0,
+                                int ksel, int append, int out_rows_stride, void* out_k, void* out_v,
+                                int32_t* seg, cudaStream_t stream, int* launches) {
+  const int vpr = d * 2 / 16;
+  const int rpb = GATHER_THREADS / vpr * GATHER_UNROLL;
+  const long long heads = static_cast<long long>(B) * Hq;
+  if (heads <= 0 || heads > 65535) return cudaErrorInvalidValue;
+  const int max_rows = (ksel < L ? ksel : L) + append;
+  const GatherStrides st = {ks.b / 8, ks.h / 8, ks.l / 8, vs.b / 8, vs.h / 8, vs.l / 8};
+  const dim3 grid(static_cast<unsigned>((max_rows + rpb - 1) / rpb > 0 ? (max_rows + rpb - 1) / rpb : 1),
+                  static_cast<unsigned>(heads));
+  const uint4* kp = static_cast<const uint4*>(k);
+  const uint4* vp = static_cast<const uint4*>(v);
+  if (vpr == 16)
+    gather_range_kernel<16><<<grid, GATHER_THREADS, 0, stream>>>(
+        kp, vp, st, idx, Hq / Hkv, Hkv, L, pos0, ksel, append, out_rows_stride,
+        static_cast<uint4*>(out_k), static_cast<uint4*>(out_v), seg);
+  else
+    gather_range_kernel<8><<<grid, GATHER_THREADS, 0, stream>>>(
+        kp, vp, st, idx, Hq / Hkv, Hkv, L, pos0, ksel, append, out_rows_stride,
+        static_cast<uint4*>(out_k), static_cast<uint4*>(out_v), seg);
+  *launches += 1;
+  return cudaGetLastError();
+}
 
 cudaError_t launch_gather(const void* k, const void* v, const KVStrides& ks, const KVStrides& vs,
                           const int32_t* idx, int B, int Hq, int Hkv, int L, int d, int W, int ksel,

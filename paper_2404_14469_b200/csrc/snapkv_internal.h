@@ -41,7 +41,8 @@ struct ScorePlan {
   int ncols;        // hpu * W
   int npad;         // ncols rounded up to 32, 64 or 128
   int tiles_stats;  // ceil(L / TILE_KEYS): the normaliser covers every key
-  int tiles_vote;   // ceil(n / TILE_KEYS): votes exist for prefix keys only
+  int n_vote;       // keys that get a vote: L - W, or what a shard of a longer prompt asks for
+  int tiles_vote;   // ceil(n_vote / TILE_KEYS): votes exist for prefix keys only
   int units_per_wave;
   int nwaves;
   int maxseg;       // partial-statistics slots per unit
@@ -93,6 +94,16 @@ struct PagedKV {
   int num_pages;         // pages in the pool; an entry outside [0, num_pages) reads as zeros
 };
 
+// A shard of a longer prompt (the positions [pos0, pos0 + L) of it).  `mask_n`: window row i
+// sees the shard's keys j <= mask_n + i (the whole prompt's prefix length minus pos0; may be
+// negative or beyond L).  With `lse_out` the statistics sweep alone runs and the shard's partial
+// natural-log sum-exp of every window row goes to lse_out [B*Hq, W] (-inf where a row sees
+// none of the shard's keys); `vote` is then not touched.
+struct ShardMode {
+  int mask_n;
+  float* lse_out;
+};
+
 struct WorkspaceLayout {
   size_t off_status, off_counters, off_partials, off_lse, off_vote, off_pooled, total;
 };
@@ -108,7 +119,8 @@ int list_schedule_items(const ScorePlan& plan, int L, int W, int Hkv, int votes_
 // waits (process-wide; one second unless snapkv_set_wait_limit_ns changed it).
 unsigned long long wait_limit_setting();
 
-bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* plan);
+// `n_vote` < 0: the keys that get a vote are the L - W prefix keys (the whole prompt is here).
+bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* plan, int n_vote = -1);
 WorkspaceLayout make_layout(const ScorePlan& p, int B, int Hq, int n, bool need_vote,
                             bool need_pooled);
 bool select_needs_scratch(int n);
@@ -127,7 +139,7 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrid
                                  int* counters, float* partials, float* lse2, cudaStream_t stream,
                                  int* launches, const float* lse_obs = nullptr,
                                  bool keep_status = false, bool never_ready = false,
-                                 const PagedKV* paged = nullptr);
+                                 const PagedKV* paged = nullptr, const ShardMode* shard = nullptr);
 
 // Pool + top-k over `rows` rows of fp32 votes.  `pooled_scratch` (select_scratch_bytes bytes)
 // is only touched when select_needs_scratch(n).  With gsum > 1 a selection row is the sum of
@@ -149,6 +161,13 @@ cudaError_t launch_gather(const void* k, const void* v, const KVStrides& ks, con
                           const int32_t* idx, int B, int Hq, int Hkv, int L, int d, int W, int ksel,
                           int out_rows_stride, void* out_k, void* out_v, cudaStream_t stream,
                           int* launches, const PagedKV* paged = nullptr);
+
+// A shard's part of the gather: rows of `idx` (global positions) that lie in [pos0, pos0 + L),
+// then `append` trailing rows of the shard; seg [B*Hq][2] = {first entry, entries} per head.
+cudaError_t launch_gather_range(const void* k, const void* v, const KVStrides& ks, const KVStrides& vs,
+                                const int32_t* idx, int B, int Hq, int Hkv, int L, int d, int pos0,
+                                int ksel, int append, int out_rows_stride, void* out_k, void* out_v,
+                                int32_t* seg, cudaStream_t stream, int* launches);
 
 cudaError_t launch_iota_idx(int32_t* out_idx, int rows, int n, int row_stride, cudaStream_t stream,
                             int* launches);

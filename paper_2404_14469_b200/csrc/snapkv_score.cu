@@ -73,6 +73,8 @@ struct ScoreArgs {
   int T1, T2;               // tiles per unit in the statistics / vote pass
   int maxseg;               // partial slots per unit
   int pipelined;            // how many waves the statistics run ahead of the votes (>= 1)
+  int mask_n;               // window row i sees keys j <= mask_n + i (n, or n minus a shard's first position)
+  int stats_only;           // 1: statistics pass alone (a shard's partial log-sum-exp), no votes
   int votes_only;           // 1: lse2 and the counters are already set, no statistics pass
   unsigned long long wait_ns;  // time limit of every device-side wait
   const int32_t* page_table;   // paged K: [batch][pages_per_seq] page numbers, else nullptr
@@ -162,10 +164,10 @@ __host__ __device__ __forceinline__ void for_each_item(const ScoreArgs& a, int c
                                                        F&& f) {
   // Phase order: statistics run `lag` waves ahead of votes: S(0) .. S(lag-1) V(0) S(lag)
   // V(1) ...; lag = 1 is the plain order S(0) V(0) S(1) V(1) ...
-  int s_next = a.votes_only ? a.nwaves : 0, v_next = 0;
-  while (v_next < a.nwaves) {
+  int s_next = a.votes_only ? a.nwaves : 0, v_next = a.stats_only ? a.nwaves : 0;
+  while (v_next < a.nwaves || s_next < a.nwaves) {
     int w, vote;
-    if (s_next < a.nwaves && s_next - v_next < lag) { w = s_next++; vote = 0; }
+    if (s_next < a.nwaves && (v_next >= a.nwaves || s_next - v_next < lag)) { w = s_next++; vote = 0; }
     else { w = v_next++; vote = 1; }
     const int u0 = w * a.upw;
     const int nu = a.upw < a.units - u0 ? a.upw : a.units - u0;
@@ -445,7 +447,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     const int rrow = 32 * q + lane;  // TMEM lane
     const int rep = rrow / NPAD;
     const int qcol = rrow - rep * NPAD;
-    const int jmax = min(a.L - 1, a.n + (qcol % a.W));  // last key window row qcol % W sees
+    const int jmax = min(a.L - 1, a.mask_n + (qcol % a.W));  // last key window row qcol % W sees
+    const int jfree = min(a.L - 1, a.mask_n);  // keys up to here are seen by every row
     const int coff = SPLIT ? wg * CPT : 0;               // first accumulator column of this thread
     const bool w16 = (a.W & 15) == 0;
     const int gpw = a.W >> 4;  // 16-column groups per head (when W is a multiple of 16)
@@ -476,7 +479,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_n(bar_te(buf), te_arrivals);
-          if (key0 + TILE_KEYS - 1 > a.n) {  // tile touches the window or the prompt's end
+          if (key0 + TILE_KEYS - 1 > jfree) {  // tile touches the window or the end of the keys
             const int kb = key0 + rep * NPAD + coff;
 #pragma unroll
             for (int ch = 0; ch < VCH; ++ch)
@@ -813,6 +816,30 @@ __global__ void lse_prep_kernel(const float* __restrict__ lse_obs, float* __rest
   if (c == 0) counters[u] = COUNTER_READY;
 }
 
+// After a statistics-only launch: folds every unit's partials, in slot order as the vote sweep
+// would, into one natural-log sum-exp per window row (counters[u] is the number of partials the
+// unit got).  One block per unit, one thread per window column.
+__global__ void lse_finish_kernel(const float* __restrict__ partials, const int* __restrict__ counters,
+                                  float* __restrict__ lse_out, int units, int maxseg, int sub_per_kv,
+                                  int g, int hpu, int W, int ncols) {
+  const int u = blockIdx.x, c = threadIdx.x;
+  if (u >= units || c >= ncols) return;
+  const int nseg = counters[u];
+  const float* pp = partials + static_cast<size_t>(u) * maxseg * MAX_COLS + c;
+  float M = -INFINITY, S = 0.f;
+  for (int sg = 0; sg < nseg; ++sg) {
+    const float pv = pp[static_cast<size_t>(sg) * MAX_COLS];
+    const float Mn = fmaxf(fmaxf(M, pv), -1e30f);
+    S = S * ex2_approx(M - Mn) + ex2_approx(pv - Mn);
+    M = Mn;
+  }
+  const int ukv = u / sub_per_kv;
+  const int hq0 = ukv * g + (u - ukv * sub_per_kv) * hpu;
+  const int hl = c / W, i = c - hl * W;
+  // log2 -> natural log; a row that saw no key of this shard has S = 0: log gives -inf
+  lse_out[static_cast<size_t>(hq0 + hl) * W + i] = (M + log2f(S)) * 0.6931471805599453f;
+}
+
 template <int D, int NCH, bool SPLIT>
 cudaError_t run_scores(const CUtensorMap& tmK, const CUtensorMap& tmQ, const ScoreArgs& a,
                        int grid, cudaStream_t stream, int* launches) {
@@ -843,7 +870,9 @@ cudaError_t run_scores(const CUtensorMap& tmK, const CUtensorMap& tmQ, const Sco
 static ScoreArgs schedule_args(const ScorePlan& plan, int L, int W, int Hkv, int votes_only) {
   ScoreArgs a = {};
   a.L = L;
-  a.n = L - W;
+  a.n = plan.n_vote;
+  a.mask_n = L - W;
+  a.stats_only = 0;
   a.W = W;
   a.Hkv = Hkv;
   a.hpu = plan.hpu;
@@ -881,8 +910,9 @@ int list_schedule_items(const ScorePlan& plan, int L, int W, int Hkv, int votes_
   return count;
 }
 
-bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* plan) {
+bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* plan, int n_vote) {
   if (B < 1 || Hq < 1 || Hkv < 1 || L < 1 || W < 1 || W > L || Hq % Hkv != 0) return false;
+  if (n_vote > L) return false;
   if (W > MAX_COLS || (d != 64 && d != 128)) return false;
   ScorePlan p;
   p.g = Hq / Hkv;
@@ -895,7 +925,8 @@ bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* pla
   p.units = static_cast<int>(units);
   p.ncols = p.hpu * W;
   p.npad = p.ncols <= 32 ? 32 : (p.ncols <= 64 ? 64 : 128);
-  const int n = L - W;
+  const int n = n_vote >= 0 ? n_vote : L - W;
+  p.n_vote = n;
   p.tiles_stats = (L + TILE_KEYS - 1) / TILE_KEYS;
   p.tiles_vote = (n + TILE_KEYS - 1) / TILE_KEYS;
   // A wave is a set of units whose keys are swept twice; with the pipelined schedule two
@@ -936,7 +967,7 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrid
                                  float* vote, int* status,
                                  int* counters, float* partials, float* lse2, cudaStream_t stream,
                                  int* launches, const float* lse_obs, bool keep_status,
-                                 bool never_ready, const PagedKV* paged) {
+                                 bool never_ready, const PagedKV* paged, const ShardMode* shard) {
   CUtensorMap tmK, tmQ;
   {
     // (d, position, KV head, batch) with the caller's strides: any layout whose rows of d
@@ -960,6 +991,10 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrid
   }
   ScoreArgs a = schedule_args(plan, L, W, Hkv, (lse_obs || never_ready) ? 1 : 0);
   a.wait_ns = wait_limit_setting();
+  if (shard) {
+    a.mask_n = shard->mask_n;
+    a.stats_only = shard->lse_out ? 1 : 0;
+  }
   a.page_table = paged ? paged->table : nullptr;
   a.pages_per_seq = paged ? paged->pages_per_seq : 0;
   a.page_size = paged ? paged->page_size : 1;
@@ -982,20 +1017,30 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrid
   const int nch = plan.npad >> 5;
   // column-split epilogue when each warpgroup's half of the columns is whole heads
   const bool split = nch >= 2 && (W % 16) == 0 && ((plan.npad / 2) % W) == 0;
+  cudaError_t e;
   if (d == 64) {
-    if (nch == 1) return run_scores<64, 1, false>(tmK, tmQ, a, grid, stream, launches);
-    if (nch == 2)
-      return split ? run_scores<64, 2, true>(tmK, tmQ, a, grid, stream, launches)
-                   : run_scores<64, 2, false>(tmK, tmQ, a, grid, stream, launches);
-    return split ? run_scores<64, 4, true>(tmK, tmQ, a, grid, stream, launches)
-                 : run_scores<64, 4, false>(tmK, tmQ, a, grid, stream, launches);
+    if (nch == 1) e = run_scores<64, 1, false>(tmK, tmQ, a, grid, stream, launches);
+    else if (nch == 2)
+      e = split ? run_scores<64, 2, true>(tmK, tmQ, a, grid, stream, launches)
+                : run_scores<64, 2, false>(tmK, tmQ, a, grid, stream, launches);
+    else
+      e = split ? run_scores<64, 4, true>(tmK, tmQ, a, grid, stream, launches)
+                : run_scores<64, 4, false>(tmK, tmQ, a, grid, stream, launches);
+  } else {
+    if (nch == 1) e = run_scores<128, 1, false>(tmK, tmQ, a, grid, stream, launches);
+    else if (nch == 2)
+      e = split ? run_scores<128, 2, true>(tmK, tmQ, a, grid, stream, launches)
+                : run_scores<128, 2, false>(tmK, tmQ, a, grid, stream, launches);
+    else
+      e = split ? run_scores<128, 4, true>(tmK, tmQ, a, grid, stream, launches)
+                : run_scores<128, 4, false>(tmK, tmQ, a, grid, stream, launches);
   }
-  if (nch == 1) return run_scores<128, 1, false>(tmK, tmQ, a, grid, stream, launches);
-  if (nch == 2)
-    return split ? run_scores<128, 2, true>(tmK, tmQ, a, grid, stream, launches)
-                 : run_scores<128, 2, false>(tmK, tmQ, a, grid, stream, launches);
-  return split ? run_scores<128, 4, true>(tmK, tmQ, a, grid, stream, launches)
-               : run_scores<128, 4, false>(tmK, tmQ, a, grid, stream, launches);
+  if (e != cudaSuccess || !a.stats_only) return e;
+  lse_finish_kernel<<<plan.units, MAX_COLS, 0, stream>>>(partials, counters, shard->lse_out, plan.units,
+                                                        plan.maxseg, plan.sub_per_kv, plan.g, plan.hpu,
+                                                        W, plan.ncols);
+  *launches += 1;
+  return cudaGetLastError();
 }
 
 }  // namespace snapkv

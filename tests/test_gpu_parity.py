@@ -144,7 +144,10 @@ def test_pool_topk_matches_oracle(rows, n, kernel, ptype, ksel):
     (2, 40960, 7, "max", 32768),
     (2, 40000, 5, "avg", 39000),
     (1, 40960, 1, "max", 40960),    # everything is kept
-    (2, 49000, 7, "max", 48000),    # generic one-CTA kernel
+    (49, 40960, 7, "max", 32767),   # enough rows for the one-CTA kernel: the same two points there
+    (49, 40960, 7, "max", 32768),
+    (49, 40000, 5, "avg", 39000),
+    (2, 49000, 17, "max", 48000),   # radius 8: generic one-CTA kernel
     (1, 70000, 5, "avg", 69000),    # many-CTA path
 ])
 def test_pool_topk_with_very_large_ksel_stays_inside_its_rows(rows, n, kernel, ptype, ksel):
