@@ -234,8 +234,18 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int gsum, int r, in
   {
     const int total = SEL_THREADS * ept;
     if (gsum == 1) {
-      for (int j = threadIdx.x; j < total; j += SEL_THREADS)
-        keys[key_slot4(j)] = (j < n) ? __float_as_uint(__ldg(vrow + j)) : 0u;
+      // eight loads in flight per thread before the first store: the votes come from L2, and
+      // one load per loop turn would pay that latency once per element (ept is a multiple of 8)
+      for (int j0 = threadIdx.x; j0 < total; j0 += 8 * SEL_THREADS) {
+        uint32_t x[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int j = j0 + u * SEL_THREADS;
+          x[u] = (j < n) ? __float_as_uint(__ldg(vrow + j)) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) keys[key_slot4(j0 + u * SEL_THREADS)] = x[u];
+      }
     } else {
       // group sum: four positions per thread and step, so that the loads of a step are
       // independent of one another; heads are added in ascending order

@@ -38,6 +38,7 @@ constexpr int CL_WARPS = CL_THREADS / 32;
 constexpr int CL_RMAX = 7;          // largest pooling radius this kernel takes
 constexpr int CL_MAX_CLUSTER = 16;  // 16 needs the non-portable cluster size
 constexpr int CL_BINS = 256;
+constexpr int CL_COPIES = 4;        // private histogram copies per CTA (two warps share one)
 
 __device__ __forceinline__ uint32_t float_to_key(float x) {
   const uint32_t b = __float_as_uint(x);
@@ -116,7 +117,7 @@ pool_topk_cluster_kernel(const float* __restrict__ vote, int n, int gsum, int r,
   constexpr int STAGED = CHUNK + 2 * CL_RMAX;
   __shared__ float raw[STAGED + STAGED / 32 + 1];
   __shared__ int hist[2][CL_BINS];        // the CTA's histogram of a round, read by the peers
-  __shared__ int hist_w[CL_WARPS][CL_BINS];  // one private histogram per warp
+  __shared__ int hist_w[CL_COPIES][CL_BINS];  // private histograms, one per pair of warps
   __shared__ int totals[CL_MAX_CLUSTER][2];  // per CTA of the cluster: keys above / equal to the threshold
   __shared__ uint32_t warp_sums[CL_WARPS];
   __shared__ uint32_t scan_total;
@@ -127,15 +128,37 @@ pool_topk_cluster_kernel(const float* __restrict__ vote, int n, int gsum, int r,
   const int c0 = static_cast<int>(rank) * CHUNK;  // first position of this CTA's chunk
   const float* vrow = vote + static_cast<size_t>(row) * gsum * n;
 
-  // ---- 1. stage the chunk and its halo: position c0 - CL_RMAX + t at slot(t); zero outside the row
-  for (int t = threadIdx.x; t < STAGED; t += CL_THREADS) {
-    const int j = c0 - CL_RMAX + t;
-    float x = 0.f;
-    if (j >= 0 && j < n) {
-      x = __ldg(vrow + j);
-      for (int g = 1; g < gsum; ++g) x += __ldg(vrow + static_cast<size_t>(g) * n + j);  // ascending head order
+  // ---- 1. stage the chunk and its halo: position c0 - CL_RMAX + t at slot(t); zero outside the row.
+  // All of a thread's loads are issued before the first value is stored: the votes come from
+  // L2, and a loop of load-then-store would pay that latency once per element.
+  {
+    float x[EPT];
+#pragma unroll
+    for (int i = 0; i < EPT; ++i) {
+      const int j = c0 + static_cast<int>(threadIdx.x) + CL_THREADS * i;
+      x[i] = (j < n) ? __ldg(vrow + j) : 0.f;
     }
-    raw[slot(t)] = x;
+    for (int g = 1; g < gsum; ++g) {  // ascending head order
+      const float* src = vrow + static_cast<size_t>(g) * n;
+#pragma unroll
+      for (int i = 0; i < EPT; ++i) {
+        const int j = c0 + static_cast<int>(threadIdx.x) + CL_THREADS * i;
+        if (j < n) x[i] += __ldg(src + j);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < EPT; ++i) raw[slot(CL_RMAX + static_cast<int>(threadIdx.x) + CL_THREADS * i)] = x[i];
+    if (threadIdx.x < 2 * CL_RMAX) {  // the halo: CL_RMAX positions before the chunk, CL_RMAX after
+      const int t = threadIdx.x < CL_RMAX ? static_cast<int>(threadIdx.x)
+                                          : CHUNK + static_cast<int>(threadIdx.x);
+      const int j = c0 - CL_RMAX + t;
+      float h = 0.f;
+      if (j >= 0 && j < n) {
+        h = __ldg(vrow + j);
+        for (int g = 1; g < gsum; ++g) h += __ldg(vrow + static_cast<size_t>(g) * n + j);
+      }
+      raw[slot(t)] = h;
+    }
   }
   __syncthreads();
 
@@ -162,22 +185,24 @@ pool_topk_cluster_kernel(const float* __restrict__ vote, int n, int gsum, int r,
   }
 
   // ---- 2. radix select, one byte per round from the top
-  // Each warp counts into a histogram of its own (pooled neighbours mostly share a bin, and
-  // in the first rounds so do most keys of the row: one shared histogram would serialise the
-  // whole CTA on a few words); thread t then adds the eight copies of bin t, publishes the
-  // sum in the CTA's histogram of this round and clears the copies for the next round.
+  // Pairs of warps count into a histogram of their own (pooled neighbours mostly share a bin,
+  // and in the first rounds so do most keys of the row: one shared histogram would serialise
+  // the whole CTA on a few words); thread t then adds the copies of bin t, publishes the sum
+  // in the CTA's histogram of this round and clears the copies for the next round.  (Shared
+  // memory per CTA decides how many 16-CTA clusters the GPU holds at once: with 44 KB it was
+  // 31, one short of the 32 rows of the 128K workload.)
   uint32_t prefix = 0u, mask = 0u;
   int krem = ksel;
   const uint32_t hist_base = smem_addr(&hist[0][0]);
   const int warp = threadIdx.x >> 5;
 #pragma unroll
-  for (int w = 0; w < CL_WARPS; ++w) hist_w[w][threadIdx.x] = 0;  // CL_BINS == CL_THREADS
+  for (int w = 0; w < CL_COPIES; ++w) hist_w[w][threadIdx.x] = 0;  // CL_BINS == CL_THREADS
   __syncthreads();
 #pragma unroll 1
   for (int round = 0; round < 4; ++round) {
     const int shift = 24 - 8 * round;
     {
-      int* h = hist_w[warp];
+      int* h = hist_w[warp % CL_COPIES];
       int cur = -1, cnt = 0;  // count runs of equal bins
 #pragma unroll
       for (int i = 0; i < EPT; ++i) {
@@ -197,7 +222,7 @@ pool_topk_cluster_kernel(const float* __restrict__ vote, int n, int gsum, int r,
     {
       int sum = 0;
 #pragma unroll
-      for (int w = 0; w < CL_WARPS; ++w) {
+      for (int w = 0; w < CL_COPIES; ++w) {
         sum += hist_w[w][threadIdx.x];
         hist_w[w][threadIdx.x] = 0;
       }
