@@ -188,9 +188,7 @@ pool_topk_cluster_kernel(const float* __restrict__ vote, int n, int gsum, int r,
   // Pairs of warps count into a histogram of their own (pooled neighbours mostly share a bin,
   // and in the first rounds so do most keys of the row: one shared histogram would serialise
   // the whole CTA on a few words); thread t then adds the copies of bin t, publishes the sum
-  // in the CTA's histogram of this round and clears the copies for the next round.  (Shared
-  // memory per CTA decides how many 16-CTA clusters the GPU holds at once: with 44 KB it was
-  // 31, one short of the 32 rows of the 128K workload.)
+  // in the CTA's histogram of this round and clears the copies for the next round.
   uint32_t prefix = 0u, mask = 0u;
   int krem = ksel;
   const uint32_t hist_base = smem_addr(&hist[0][0]);
