@@ -378,8 +378,9 @@ def snapkv_gather_range(k_shard, v_shard, idx, pos0: int, append: int):
     B, Hkv, Ls, d = k_shard.shape
     _, Hq, ksel = idx.shape
     rows = min(ksel, Ls) + append
-    out_k = torch.zeros(B, Hq, rows, d, dtype=torch.bfloat16, device=k_shard.device)
-    out_v = torch.zeros_like(out_k)
+    # rows behind a head's segment (and its appended rows) are left as allocated
+    out_k = torch.empty(B, Hq, rows, d, dtype=torch.bfloat16, device=k_shard.device)
+    out_v = torch.empty_like(out_k)
     seg = torch.empty(B, Hq, 2, dtype=torch.int32, device=k_shard.device)
     code = lib().snapkv_gather_range(k_shard.data_ptr(), v_shard.data_ptr(), idx.data_ptr(), B, Hq, Hkv, Ls, d,
                                      int(pos0), ksel, int(append), out_k.data_ptr(), out_v.data_ptr(), rows,

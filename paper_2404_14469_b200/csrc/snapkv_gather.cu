@@ -105,38 +105,43 @@ gather_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v, const Ga
 }
 
 // A shard of a longer prompt holds positions [pos0, pos0 + L).  Of a head's ascending list of
-// selected positions, the entries inside that range form one contiguous segment; this kernel
-// finds it (two binary searches per block) and copies those rows, then `append` trailing rows
-// of the shard (the window rows, on the shard that holds them), into rows [0, count + append)
-// of the head's output.  seg[head] = {first entry of the segment, entries in it}.
+// selected positions, the entries inside that range form one contiguous segment.
+// seg_kernel finds it, one thread per head (two binary searches): seg[head] = {first entry of
+// the segment, entries in it}.  gather_range_kernel then copies those rows and `append`
+// trailing rows of the shard (the window rows, on the shard that holds them) into rows
+// [0, count + append) of the head's output.
+__global__ void seg_kernel(const int32_t* __restrict__ idx, int heads, int ksel, int pos0, int L,
+                           int32_t* __restrict__ seg) {
+  const int bh = blockIdx.x * blockDim.x + threadIdx.x;
+  if (bh >= heads) return;
+  const int32_t* idx_head = idx + static_cast<size_t>(bh) * ksel;
+  auto lower_bound = [&](int value) {  // first entry >= value
+    int lo = 0, hi = ksel;
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (__ldg(idx_head + mid) < value) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+  };
+  const int lo = lower_bound(pos0);
+  seg[2 * bh] = lo;
+  seg[2 * bh + 1] = lower_bound(pos0 + L) - lo;
+}
+
 template <int VPR>
 __global__ void __launch_bounds__(GATHER_THREADS, GATHER_MIN_BLOCKS)
 gather_range_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v, const GatherStrides st,
                     const int32_t* __restrict__ idx, int g, int Hkv, int L, int pos0, int ksel, int append,
                     int out_stride, uint4* __restrict__ out_k, uint4* __restrict__ out_v,
-                    int32_t* __restrict__ seg) {
+                    const int32_t* __restrict__ seg) {
   constexpr int RPT = GATHER_THREADS / VPR;
   constexpr int RPB = RPT * GATHER_UNROLL;
   __shared__ int s_lo, s_cnt;
   const int bh = blockIdx.y;
   const int32_t* idx_head = idx + static_cast<size_t>(bh) * ksel;
   if (threadIdx.x == 0) {
-    auto lower_bound = [&](int value) {  // first entry >= value
-      int lo = 0, hi = ksel;
-      while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (__ldg(idx_head + mid) < value) lo = mid + 1; else hi = mid;
-      }
-      return lo;
-    };
-    const int lo = lower_bound(pos0);
-    const int hi = lower_bound(pos0 + L);
-    s_lo = lo;
-    s_cnt = hi - lo;
-    if (blockIdx.x == 0) {
-      seg[2 * bh] = lo;
-      seg[2 * bh + 1] = hi - lo;
-    }
+    s_lo = __ldg(seg + 2 * bh);
+    s_cnt = __ldg(seg + 2 * bh + 1);
   }
   __syncthreads();
   const int lo = s_lo, cnt = s_cnt;
@@ -177,6 +182,9 @@ cudaError_t launch_gather_range(const void* k, const void* v, const KVStrides& k
   const GatherStrides st = {ks.b / 8, ks.h / 8, ks.l / 8, vs.b / 8, vs.h / 8, vs.l / 8};
   const dim3 grid(static_cast<unsigned>((max_rows + rpb - 1) / rpb > 0 ? (max_rows + rpb - 1) / rpb : 1),
                   static_cast<unsigned>(heads));
+  seg_kernel<<<static_cast<unsigned>((heads + 127) / 128), 128, 0, stream>>>(idx, static_cast<int>(heads), ksel,
+                                                                             pos0, L, seg);
+  *launches += 1;
   const uint4* kp = static_cast<const uint4*>(k);
   const uint4* vp = static_cast<const uint4*>(v);
   if (vpr == 16)
