@@ -217,6 +217,7 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int gsum, int r, in
   __shared__ int warp_sums[SEL_WARPS];
   __shared__ int scan_total;
   __shared__ int sel_bin, sel_above, sel_count, ncand_s;
+  __shared__ int above_s, br_lo, br_hi;
   __shared__ uint32_t red_min[SEL_WARPS], red_max[SEL_WARPS];
   __shared__ uint32_t cand[CAND_CAP];
   int ncand = 0;
@@ -354,6 +355,107 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int gsum, int r, in
     if (shift < 0) shift = 0;
     uint32_t width_m1 = range;  // candidates are keys with key - lo <= width_m1
     bool first = true;
+    // 2a. A guess from a sample.  Every fourth key goes into the histogram (a quarter of the
+    // shared-memory atomics of a full pass, which is what that pass spends its time on); the
+    // sample's cumulative counts give a RANGE of bins that should hold the ksel-th key: the
+    // bins between the sample ranks 4 standard deviations to either side of ksel/4.  One sweep
+    // then counts, exactly, the keys above that range and collects the keys inside it.  If the
+    // exact counts confirm that the ksel-th key is inside and the range fits the candidate list,
+    // the threshold is refined on the list; otherwise nothing of this is used and the full
+    // histogram pass below decides (exactness never rests on the sample).
+    {
+      for (int b = threadIdx.x; b < NBINS; b += SEL_THREADS) hist[b] = 0;
+      if (threadIdx.x == 0) { ncand_s = 0; above_s = 0; br_lo = 0; br_hi = NBINS - 1; }
+      __syncthreads();
+      for (int i0 = 0; i0 < ept; i0 += 4) {
+        const uint32_t key = keys[key_slot4(base + i0)];
+        if (key >= kmin) atomicAdd(&hist[(key - kmin) >> shift], 1);  // (padding keys are below kmin)
+      }
+      __syncthreads();
+      int c0 = 0, c1 = 0;
+      const int b0 = NBINS - 1 - 2 * static_cast<int>(threadIdx.x);
+      if (b0 >= 0) c0 = hist[b0];
+      if (b0 - 1 >= 0) c1 = hist[b0 - 1];
+      const int before = block_exclusive_scan(c0 + c1, warp_sums, &scan_total);
+      const int m_s = scan_total;  // samples in the row
+      const float pfrac = static_cast<float>(ksel) / static_cast<float>(n);
+      const int delta = static_cast<int>(4.f * sqrtf(static_cast<float>(m_s) * pfrac * (1.f - pfrac))) + 2;
+      const int r_mid = static_cast<int>(static_cast<long long>(ksel) * m_s / n);
+      const int r_hi = max(1, r_mid - delta);  // sample rank that bounds the range from above
+      const int r_lo = r_mid + delta;          // ... from below; beyond the sample: down to the lowest bin
+      if (c0 > 0 && before < r_hi && r_hi <= before + c0) br_hi = b0;
+      else if (c1 > 0 && before + c0 < r_hi && r_hi <= before + c0 + c1) br_hi = b0 - 1;
+      if (c0 > 0 && before < r_lo && r_lo <= before + c0) br_lo = b0;
+      else if (c1 > 0 && before + c0 < r_lo && r_lo <= before + c0 + c1) br_lo = b0 - 1;
+      __syncthreads();
+      const int b_hi = br_hi, b_lo = r_lo > m_s ? 0 : br_lo;
+      int cntg = 0, cnti = 0;
+      for (int i0 = 0; i0 < ept; i0 += 4) {
+        const uint4 kv = ld_keys4(keys, base + i0);
+        const uint32_t k4[4] = {kv.x, kv.y, kv.z, kv.w};
+        uint32_t bg = 0u, bi = 0u;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const uint32_t key = k4[u];
+          const int bin = static_cast<int>((key - kmin) >> shift);
+          const bool real = key >= kmin;
+          const bool gt = real && bin > b_hi;
+          const bool inb = real && bin >= b_lo && bin <= b_hi;
+          bg |= static_cast<uint32_t>(gt) << u;
+          bi |= static_cast<uint32_t>(inb) << u;
+          cntg += gt;
+          cnti += inb;
+        }
+        if (i0 < 32) { m_gt[0] |= bg << i0; m_in[0] |= bi << i0; }
+        else { m_gt[1] |= bg << (i0 - 32); m_in[1] |= bi << (i0 - 32); }
+      }
+      // the keys inside the range go to the candidate list: one atomic per warp reserves the
+      // warp's slots (a thousand single appends to one counter would take as long as the pass
+      // this replaces), a warp scan places each thread's keys
+      {
+        int inc = cnti;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += y;
+        }
+        int wbase = 0;
+        if (lane == 31 && inc > 0) wbase = atomicAdd(&ncand_s, inc);
+        wbase = __shfl_sync(0xffffffffu, wbase, 31);
+        int at = wbase + inc - cnti;
+#pragma unroll
+        for (int wd = 0; wd < MASK_WORDS; ++wd) {
+          uint32_t rest = m_in[wd];
+          while (rest) {
+            const int i = wd * 32 + __ffs(rest) - 1;
+            rest &= rest - 1;
+            if (at < CAND_CAP) cand[at] = keys[key_slot4(base + i)];
+            ++at;
+          }
+        }
+      }
+      cntg = __reduce_add_sync(0xffffffffu, cntg);
+      if (lane == 0 && cntg) atomicAdd(&above_s, cntg);
+      __syncthreads();
+      const int above = above_s, inside = ncand_s;
+      __syncthreads();  // everybody has read the counts before anybody starts the next pass
+      if (above < ksel && ksel <= above + inside && inside <= CAND_CAP) {
+        first = false;
+        use_list = true;
+        ncand = inside;
+        krem = ksel - above;
+        lo = kmin + (static_cast<uint32_t>(b_lo) << shift);
+        const unsigned long long top =
+            static_cast<unsigned long long>(kmin) + (static_cast<unsigned long long>(b_hi + 1) << shift) - 1ull;
+        const uint32_t hi_key = top > kmax ? kmax : static_cast<uint32_t>(top);
+        width_m1 = hi_key - lo;
+        shift = 32 - __clz(width_m1 | 1u) - 11;
+        if (shift < 0) shift = 0;
+      } else {
+#pragma unroll
+        for (int wd = 0; wd < MASK_WORDS; ++wd) { m_gt[wd] = 0u; m_in[wd] = 0u; }
+      }
+    }
 #pragma unroll 1
     for (;;) {
       for (int b = threadIdx.x; b < NBINS; b += SEL_THREADS) hist[b] = 0;
