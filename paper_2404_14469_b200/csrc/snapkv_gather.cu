@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "launch.cuh"
 #include "snapkv_internal.h"
 
 namespace snapkv {
@@ -53,6 +54,7 @@ gather_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v, const Ga
               int W, int ksel, int out_stride, uint4* __restrict__ out_k, uint4* __restrict__ out_v) {
   constexpr int RPT = GATHER_THREADS / VPR;      // rows covered by the block per unrolled step
   constexpr int RPB = RPT * GATHER_UNROLL;       // rows per block
+  pdl_wait();  // launched early behind the select kernel: idx is complete only from here on
   const int rows = ksel + W;
   const int n = L - W;
   const int bh = h0 + blockIdx.y;
@@ -218,30 +220,31 @@ cudaError_t launch_gather(const void* k, const void* v, const KVStrides& ks, con
   const unsigned gx = static_cast<unsigned>((rows + rpb - 1) / rpb);
   // blockIdx.y is limited to 65535: go through the heads in slabs if there are more
   const long long slab = 65535;
-  for (long long h0 = 0; h0 < heads; h0 += slab) {
+  cudaError_t e = cudaSuccess;
+  for (long long h0 = 0; h0 < heads && e == cudaSuccess; h0 += slab) {
     const unsigned gy = static_cast<unsigned>(heads - h0 < slab ? heads - h0 : slab);
     const int h0i = static_cast<int>(h0);
     const dim3 grid(gx, gy);
     if (paged) {
       const GatherPages pg = {paged->table, paged->pages_per_seq, paged->page_size, paged->num_pages};
       if (vpr == 16)
-        gather_kernel<16, true><<<grid, GATHER_THREADS, 0, stream>>>(
-            kp, vp, st, pg, idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
+        e = launch_pdl(gather_kernel<16, true>, grid, dim3(GATHER_THREADS), 0, stream, kp, vp, st, pg,
+                       idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
       else
-        gather_kernel<8, true><<<grid, GATHER_THREADS, 0, stream>>>(
-            kp, vp, st, pg, idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
+        e = launch_pdl(gather_kernel<8, true>, grid, dim3(GATHER_THREADS), 0, stream, kp, vp, st, pg,
+                       idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
     } else {
       const GatherPages pg = {nullptr, 0, 1, 0};
       if (vpr == 16)
-        gather_kernel<16, false><<<grid, GATHER_THREADS, 0, stream>>>(
-            kp, vp, st, pg, idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
+        e = launch_pdl(gather_kernel<16, false>, grid, dim3(GATHER_THREADS), 0, stream, kp, vp, st, pg,
+                       idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
       else
-        gather_kernel<8, false><<<grid, GATHER_THREADS, 0, stream>>>(
-            kp, vp, st, pg, idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
+        e = launch_pdl(gather_kernel<8, false>, grid, dim3(GATHER_THREADS), 0, stream, kp, vp, st, pg,
+                       idx, h0i, g, Hkv, L, W, ksel, out_rows_stride, okp, ovp);
     }
     *launches += 1;
   }
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace snapkv

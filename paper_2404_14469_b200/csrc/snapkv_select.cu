@@ -15,6 +15,7 @@
 #include <stdint.h>
 
 #include "../../include/snapkv.h"
+#include "launch.cuh"
 #include "snapkv_internal.h"
 
 namespace snapkv {
@@ -226,6 +227,8 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int gsum, int r, in
   const float* vrow = vote + static_cast<size_t>(row) * gsum * n;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int base = threadIdx.x * ept;
+  // the gather kernel behind this one may become resident now; it waits for this kernel's end
+  pdl_launch_dependents();
 
   // ---- 1. pooling
   // The row is first copied into the key slots with coalesced loads (raw fp32 bits), then
