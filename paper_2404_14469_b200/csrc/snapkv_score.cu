@@ -173,7 +173,11 @@ __host__ __device__ __forceinline__ void for_each_item(const ScoreArgs& a, int c
     const int nu = a.upw < a.units - u0 ? a.upw : a.units - u0;
     const int T = vote ? a.T2 : a.T1;
     const long long TT = static_cast<long long>(nu) * T;
-    const long long lo = part_lo(cta, TT, G), hi = part_lo(cta + 1, TT, G);
+    // TT is seldom a multiple of G, so some CTAs get one tile less than the others; which
+    // ones moves on by one CTA from phase to phase, so that over the phases of a launch no
+    // CTA carries the longer share every time
+    const int cr = (cta + 2 * w + vote) % G;
+    const long long lo = part_lo(cr, TT, G), hi = part_lo(cr + 1, TT, G);
     for (long long pos = lo; pos < hi;) {
       const int ul = static_cast<int>(pos / T);
       Item it;
@@ -188,7 +192,7 @@ __host__ __device__ __forceinline__ void for_each_item(const ScoreArgs& a, int c
       if (TT1 >= G) {  // every CTA has tiles: a unit's owners are consecutive CTAs
         const int cfirst = cta_of_tile(static_cast<long long>(ul) * a.T1, TT1, G);
         const int clast = cta_of_tile(static_cast<long long>(ul + 1) * a.T1 - 1, TT1, G);
-        it.slot = cta - cfirst;
+        it.slot = cr - cfirst;
         it.nseg = clast - cfirst + 1;
       } else {         // fewer tiles than CTAs: one tile per owner, one partial per tile
         it.slot = it.t0;
