@@ -150,15 +150,48 @@ struct Item {
   int unit, t0, t1, vote, slot, nseg;
 };
 
-// CTA `c` of `G` owns tiles [c*TT/G, (c+1)*TT/G) of a phase's TT tiles.
-__host__ __device__ __forceinline__ long long part_lo(long long c, long long TT, int G) { return c * TT / G; }
-// the CTA whose range contains tile x: the largest c with part_lo(c) <= x
-__host__ __device__ __forceinline__ int cta_of_tile(long long x, long long TT, int G) {
-  return static_cast<int>(((x + 1) * G + TT - 1) / TT) - 1;
+// The work items of CTA `cr` in one phase: the phase's TT = nu * T tiles (units u0 .. u0+nu-1,
+// T tiles each) are cut into G consecutive shares, CTA c owning tiles [c*TT/G, (c+1)*TT/G); a
+// share that crosses a unit boundary is one item per unit.  I is the integer type of the tile
+// arithmetic: every warp of a CTA walks the list, at every item, so the divisions are done in
+// 32 bits whenever the products fit (64-bit divisions cost about 0.1 us each here).
+template <typename I, typename F>
+__host__ __device__ __forceinline__ bool phase_items(const ScoreArgs& a, int cr, int G, int u0,
+                                                     int nu, int T, int vote, F&& f) {
+  const I g = static_cast<I>(G);
+  const I TT = static_cast<I>(nu) * static_cast<I>(T);
+  const I lo = static_cast<I>(cr) * TT / g, hi = static_cast<I>(cr + 1) * TT / g;
+  // where this CTA's partial of a unit goes and how many partials the unit gets follow from
+  // the statistics-pass partition of the unit's wave (TT1 tiles)
+  const I T1 = static_cast<I>(a.T1);
+  const I TT1 = static_cast<I>(nu) * T1;
+  // the CTA whose share contains tile x: the largest c with c*TT1/G <= x
+  auto cta_of_tile = [&](I x) { return static_cast<int>(((x + 1) * g + TT1 - 1) / TT1) - 1; };
+  for (I pos = lo; pos < hi;) {
+    const I ul = pos / static_cast<I>(T);
+    Item it;
+    it.unit = u0 + static_cast<int>(ul);
+    it.t0 = static_cast<int>(pos - ul * static_cast<I>(T));
+    const I t1 = static_cast<I>(it.t0) + (hi - pos);
+    it.t1 = t1 < static_cast<I>(T) ? static_cast<int>(t1) : T;
+    it.vote = vote;
+    if (TT1 >= g) {  // every CTA has tiles: a unit's owners are consecutive CTAs
+      const int cfirst = cta_of_tile(ul * T1);
+      const int clast = cta_of_tile((ul + 1) * T1 - 1);
+      it.slot = cr - cfirst;
+      it.nseg = clast - cfirst + 1;
+    } else {         // fewer tiles than CTAs: one tile per owner, one partial per tile
+      it.slot = it.t0;
+      it.nseg = a.T1;
+    }
+    pos += static_cast<I>(it.t1 - it.t0);
+    if (!f(it)) return false;
+  }
+  return true;
 }
 
 // Calls f(item) for every work item of this CTA in schedule order; stops when f
-// returns false.  All three warp roles walk the same list.
+// returns false.  All warp roles walk the same list.
 template <typename F>
 __host__ __device__ __forceinline__ void for_each_item(const ScoreArgs& a, int cta, int G, int lag,
                                                        F&& f) {
@@ -172,35 +205,15 @@ __host__ __device__ __forceinline__ void for_each_item(const ScoreArgs& a, int c
     const int u0 = w * a.upw;
     const int nu = a.upw < a.units - u0 ? a.upw : a.units - u0;
     const int T = vote ? a.T2 : a.T1;
-    const long long TT = static_cast<long long>(nu) * T;
     // TT is seldom a multiple of G, so some CTAs get one tile less than the others; which
     // ones moves on by one CTA from phase to phase, so that over the phases of a launch no
     // CTA carries the longer share every time
     const int cr = (cta + 2 * w + vote) % G;
-    const long long lo = part_lo(cr, TT, G), hi = part_lo(cr + 1, TT, G);
-    for (long long pos = lo; pos < hi;) {
-      const int ul = static_cast<int>(pos / T);
-      Item it;
-      it.unit = u0 + ul;
-      it.t0 = static_cast<int>(pos - static_cast<long long>(ul) * T);
-      const long long t1 = it.t0 + (hi - pos);
-      it.t1 = static_cast<int>(t1 < T ? t1 : T);
-      it.vote = vote;
-      // where this CTA's partial of the unit goes / how many partials the unit gets:
-      // both follow from the statistics-pass partition of the unit's wave
-      const long long TT1 = static_cast<long long>(nu) * a.T1;
-      if (TT1 >= G) {  // every CTA has tiles: a unit's owners are consecutive CTAs
-        const int cfirst = cta_of_tile(static_cast<long long>(ul) * a.T1, TT1, G);
-        const int clast = cta_of_tile(static_cast<long long>(ul + 1) * a.T1 - 1, TT1, G);
-        it.slot = cr - cfirst;
-        it.nseg = clast - cfirst + 1;
-      } else {         // fewer tiles than CTAs: one tile per owner, one partial per tile
-        it.slot = it.t0;
-        it.nseg = a.T1;
-      }
-      pos += it.t1 - it.t0;
-      if (!f(it)) return;
-    }
+    const long long tmax = static_cast<long long>(nu) * (a.T1 > T ? a.T1 : T);
+    const bool fits32 = (tmax + 1) * (G + 1) < (1ll << 32);
+    const bool go_on = fits32 ? phase_items<uint32_t>(a, cr, G, u0, nu, T, vote, f)
+                              : phase_items<unsigned long long>(a, cr, G, u0, nu, T, vote, f);
+    if (!go_on) return;
   }
 }
 
