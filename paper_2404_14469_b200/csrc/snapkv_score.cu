@@ -946,11 +946,16 @@ bool make_score_plan(int B, int Hq, int Hkv, int L, int d, int W, ScorePlan* pla
   p.n_vote = n;
   p.tiles_stats = (L + TILE_KEYS - 1) / TILE_KEYS;
   p.tiles_vote = (n + TILE_KEYS - 1) / TILE_KEYS;
-  // A wave is a set of units whose keys are swept twice; with the pipelined schedule two
-  // waves are live in L2 at a time, so a wave holds about 32 MiB of keys.  Units too big
-  // for that take the sequential schedule, one unit per wave.
+  // A wave is a set of units whose keys are swept twice, WAVE_BYTES of keys; the statistics
+  // run WAVE_LAG waves ahead of the votes.  Units too big for a wave take one wave each.
   const long long kbytes = static_cast<long long>(L) * d * 2;
-  long long kv_per_wave = (WAVE_BYTES) / kbytes;
+  // With 128 window columns on one unit per KV head a vote tile costs the same from L2 as from
+  // HBM (the softmax warps are its bound), so nothing is lost by waves too big for L2, and fewer,
+  // longer phases split more evenly over the CTAs: such shapes take waves of twice the size
+  // (191.6 vs 193.6 us per layer on the 32K GQA workload; narrower units and KV heads with
+  // two sub-groups, whose vote tiles do gain from L2, are 3-5 % slower that way).
+  const long long wave_bytes = (p.ncols == 128 && p.sub_per_kv == 1) ? 2 * WAVE_BYTES : WAVE_BYTES;
+  long long kv_per_wave = wave_bytes / kbytes;
   // units bigger than a wave run one per wave: their second sweep comes from HBM, but the
   // statistics of the next unit still hide the hand-over between the two passes
   p.pipelined = WAVE_LAG;
