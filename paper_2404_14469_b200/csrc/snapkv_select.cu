@@ -650,6 +650,7 @@ __device__ __forceinline__ void wide_histogram(const uint32_t (&key_of_thread)[3
 __global__ void __launch_bounds__(WIDE_THREADS)
 wide_pool_kernel(const float* __restrict__ vote, int n, int gsum, int pool_kernel, int pool_type,
                  WideBufs wb) {
+  pdl_launch_dependents();  // the kernels behind this one are launched early and wait for its end
   __shared__ float raw[WIDE_CHUNK + 2 * WIDE_HALO + (WIDE_CHUNK + 2 * WIDE_HALO) / 32 + 1];
   __shared__ int hist_s[NBINS];
   const int row = blockIdx.y;
@@ -690,6 +691,8 @@ wide_pool_kernel(const float* __restrict__ vote, int n, int gsum, int pool_kerne
 // threshold, clear the histogram for the next pass.
 __global__ void __launch_bounds__(SEL_THREADS)
 wide_pick_kernel(int pass, int ksel, WideBufs wb) {
+  pdl_launch_dependents();
+  pdl_wait();  // launched early: the previous kernel's results are complete only from here on
   __shared__ int warp_sums[SEL_WARPS];
   __shared__ int scan_total;
   const int row = blockIdx.x;
@@ -719,6 +722,8 @@ wide_pick_kernel(int pass, int ksel, WideBufs wb) {
 
 __global__ void __launch_bounds__(WIDE_THREADS)
 wide_hist_kernel(int n, int pass, WideBufs wb) {
+  pdl_launch_dependents();
+  pdl_wait();  // launched early: the previous kernel's results are complete only from here on
   __shared__ int hist_s[NBINS];
   const int row = blockIdx.y;
   // lane-strided reads (coalesced); the order of the keys does not matter here.  Only keys
@@ -748,6 +753,8 @@ wide_hist_kernel(int n, int pass, WideBufs wb) {
 // Per chunk: how many keys are above the threshold and how many equal it.
 __global__ void __launch_bounds__(WIDE_THREADS)
 wide_count_kernel(int n, WideBufs wb) {
+  pdl_launch_dependents();
+  pdl_wait();  // launched early: the previous kernel's results are complete only from here on
   __shared__ int sg, se;
   const int row = blockIdx.y;
   if (threadIdx.x == 0) { sg = 0; se = 0; }
@@ -780,6 +787,8 @@ wide_count_kernel(int n, WideBufs wb) {
 // to it until ksel positions are out, in ascending position.
 __global__ void __launch_bounds__(WIDE_THREADS)
 wide_write_kernel(int n, int ksel, int32_t* __restrict__ out_idx, WideBufs wb) {
+  pdl_launch_dependents();
+  pdl_wait();  // launched early: the previous kernel's results are complete only from here on
   __shared__ int warp_sums[WIDE_THREADS / 32];
   const int row = blockIdx.y;
   const uint32_t T = static_cast<uint32_t>(wb.state[row * 8 + 0]);
@@ -940,13 +949,18 @@ cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel
   if (e != cudaSuccess) return e;
   const dim3 grid(wb.nblk, rows);
   wide_pool_kernel<<<grid, WIDE_THREADS, 0, stream>>>(vote, n, gsum, pool_kernel, pool_type, wb);
-  wide_pick_kernel<<<rows, SEL_THREADS, 0, stream>>>(0, ksel, wb);
-  wide_hist_kernel<<<grid, WIDE_THREADS, 0, stream>>>(n, 1, wb);
-  wide_pick_kernel<<<rows, SEL_THREADS, 0, stream>>>(1, ksel, wb);
-  wide_hist_kernel<<<grid, WIDE_THREADS, 0, stream>>>(n, 2, wb);
-  wide_pick_kernel<<<rows, SEL_THREADS, 0, stream>>>(2, ksel, wb);
-  wide_count_kernel<<<grid, WIDE_THREADS, 0, stream>>>(n, wb);
-  wide_write_kernel<<<grid, WIDE_THREADS, 0, stream>>>(n, ksel, out_idx, wb);
+  // the seven kernels behind the first are launched with programmatic dependent launch:
+  // each becomes resident while its predecessor runs and waits for it before its first read
+  const dim3 one(rows), st(SEL_THREADS), wt(WIDE_THREADS);
+  e = cudaGetLastError();
+  if (e == cudaSuccess) e = launch_pdl(wide_pick_kernel, one, st, 0, stream, 0, ksel, wb);
+  if (e == cudaSuccess) e = launch_pdl(wide_hist_kernel, grid, wt, 0, stream, n, 1, wb);
+  if (e == cudaSuccess) e = launch_pdl(wide_pick_kernel, one, st, 0, stream, 1, ksel, wb);
+  if (e == cudaSuccess) e = launch_pdl(wide_hist_kernel, grid, wt, 0, stream, n, 2, wb);
+  if (e == cudaSuccess) e = launch_pdl(wide_pick_kernel, one, st, 0, stream, 2, ksel, wb);
+  if (e == cudaSuccess) e = launch_pdl(wide_count_kernel, grid, wt, 0, stream, n, wb);
+  if (e == cudaSuccess) e = launch_pdl(wide_write_kernel, grid, wt, 0, stream, n, ksel, out_idx, wb);
+  if (e != cudaSuccess) return e;
   *launches += 8;
   return cudaGetLastError();
 }
