@@ -34,7 +34,11 @@
  *     side stream and events among all calls on a device: one caller per device at a
  *     time.
  *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
- *     default stream).  Calls return without synchronising unless stated.
+ *     default stream).  Calls return without synchronising unless stated.  Several of
+ *     the kernels are launched with programmatic dependent launch: their blocks may
+ *     become resident while the stream's previous kernel - the caller's included - is
+ *     still running, but they read and write nothing before that kernel has completed
+ *     and its writes are visible, so stream order holds for every buffer.
  *   - Errors come back as a snapkv_status_t; nothing aborts or throws.  Argument
  *     errors are found on the host before anything is launched.
  *   - A device-side wait that exceeds its time limit stops the kernel early and
