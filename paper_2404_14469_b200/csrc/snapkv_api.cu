@@ -316,7 +316,7 @@ static snapkv_status_t compress_impl(const void* q_obs, const void* k, const voi
     return SNAPKV_ERR_CUDA;
   if (launch_pool_topk(vote, B * Ho, n, pool_kernel, pool_type, ksel, out_idx,
                        scratch ? reinterpret_cast<float*>(ws + w.off_pooled) : nullptr, s,
-                       &launches, gsum) != cudaSuccess)
+                       &launches, gsum, /*vote_is_scratch=*/true) != cudaSuccess)
     return SNAPKV_ERR_CUDA;
   if (launch_gather(k, v, ks, vs, out_idx, B, Ho, Hkv, L, d, W, ksel, budget, out_k, out_v, s,
                     &launches, paged) != cudaSuccess)

@@ -144,10 +144,12 @@ cudaError_t launch_window_scores(const void* q_obs, const void* k, const KVStrid
 // Pool + top-k over `rows` rows of fp32 votes.  `pooled_scratch` (select_scratch_bytes bytes)
 // is only touched when select_needs_scratch(n).  With gsum > 1 a selection row is the sum of
 // gsum consecutive rows of `vote` (which then holds rows * gsum rows): the query heads of a
-// group selecting together.
+// group selecting together.  vote_is_scratch: nobody reads `vote` after this call, so a
+// kernel may leave its contents undefined (dirty L2 lines dropped instead of written back).
 cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel, int pool_type,
                              int ksel, int32_t* out_idx, float* pooled_scratch,
-                             cudaStream_t stream, int* launches, int gsum = 1);
+                             cudaStream_t stream, int* launches, int gsum = 1,
+                             bool vote_is_scratch = false);
 
 // The one-cluster-per-row select kernel: whether it takes rows of this length and pooling
 // kernel on the current device, and its launch (same contract as launch_pool_topk, no scratch).

@@ -22,6 +22,12 @@ namespace snapkv {
 
 namespace {
 
+// Tells L2 that a 128-byte line (global memory, 128-byte aligned) holds nothing worth keeping:
+// a dirty line may then be dropped instead of written back.  Its contents are undefined afterwards.
+__device__ __forceinline__ void discard_l2_line(const void* p) {
+  asm volatile("discard.global.L2 [%0], 128;" ::"l"(__cvta_generic_to_global(p)) : "memory");
+}
+
 constexpr int SEL_THREADS = 1024;
 constexpr int SEL_WARPS = SEL_THREADS / 32;
 constexpr int SEL_SMEM_KEYS = 49152;  // rows up to this length keep their keys on chip
@@ -212,7 +218,7 @@ constexpr int MASK_WORDS = 2;    // a thread owns at most 64 positions (SEL_SMEM
 template <int RMAX, int PT>
 __global__ void __launch_bounds__(SEL_THREADS, 1)
 pool_topk_fast_kernel(const float* __restrict__ vote, int n, int gsum, int r, int pool_type,
-                      int ept, int ksel, int32_t* __restrict__ out_idx) {
+                      int ept, int ksel, int32_t* __restrict__ out_idx, int discard_votes) {
   extern __shared__ __align__(16) uint32_t keys[];
   __shared__ int hist[NBINS];
   __shared__ int warp_sums[SEL_WARPS];
@@ -271,6 +277,17 @@ pool_topk_fast_kernel(const float* __restrict__ vote, int n, int gsum, int r, in
       }
     }
     __syncthreads();
+    if (discard_votes && gsum == 1) {
+      // The row is in shared memory and its votes are scratch that nobody reads again: drop the
+      // whole 128-byte lines inside the row from L2, so that they are not written back to HBM
+      // while the gather kernel needs the bandwidth (16.8 MB per layer of the 32K GQA workload).
+      // Lines that the row shares with its neighbours stay.
+      const uintptr_t b0 = (reinterpret_cast<uintptr_t>(vrow) + 127) & ~static_cast<uintptr_t>(127);
+      const uintptr_t b1 = reinterpret_cast<uintptr_t>(vrow + n) & ~static_cast<uintptr_t>(127);
+      for (uintptr_t a = b0 + static_cast<uintptr_t>(threadIdx.x) * 128; a < b1;
+           a += static_cast<uintptr_t>(SEL_THREADS) * 128)
+        discard_l2_line(reinterpret_cast<const void*>(a));
+    }
     // a[]: the last RMAX values before the current block of 8, the block, the next block
     float a[RMAX + 16];
     float halo_r[RMAX > 0 ? RMAX : 1];
@@ -882,7 +899,7 @@ size_t select_scratch_bytes(int rows, int n) {
 
 cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel, int pool_type,
                              int ksel, int32_t* out_idx, float* pooled_scratch,
-                             cudaStream_t stream, int* launches, int gsum) {
+                             cudaStream_t stream, int* launches, int gsum, bool vote_is_scratch) {
   // the opt-in to more than 48 KB of dynamic shared memory is a property of the device's
   // context, so it is made once per device
   DeviceOnce& once = select_attr_once();
@@ -915,7 +932,8 @@ cudaError_t launch_pool_topk(const float* vote, int rows, int n, int pool_kernel
     const int words = key_slot4_host(SEL_THREADS * ept) + 4;
 #define SNAPKV_FAST_LAUNCH(RM, P)                                                            \
   pool_topk_fast_kernel<RM, P><<<rows, SEL_THREADS, words * 4, stream>>>(vote, n, gsum, r,    \
-                                                                        pool_type, ept, ksel, out_idx)
+                                                                        pool_type, ept, ksel, out_idx, \
+                                                                        vote_is_scratch ? 1 : 0)
     // the paper's kernel sizes 5, 7 and 13 have instantiations of their own
     const bool mx = pool_type == 0;
     if (r == 2) { if (mx) SNAPKV_FAST_LAUNCH(2, 0); else SNAPKV_FAST_LAUNCH(2, 1); }
