@@ -191,6 +191,26 @@ def test_pool_topk_exact_ties_take_lower_positions(n, ksel):
     assert np.array_equal(idx[1], orc.topk_positions(pooled, ksel))
 
 
+@pytest.mark.parametrize("rows,n,kernel,ptype,ksel", [
+    (128, 32736, 5, "avg", 4064),    # the one-CTA kernel, the benchmarked shape
+    (8, 16352, 7, "max", 992),       # the cluster kernel
+    (2, 200000, 7, "max", 2048),     # the many-launch path
+])
+def test_pool_topk_leaves_the_callers_votes_alone(rows, n, kernel, ptype, ksel):
+    # the whole-step calls let the select kernel drop their scratch votes from L2 once read;
+    # votes that the caller hands to the staged call are the caller's and must come back intact,
+    # also after a second call on the same tensor
+    g = torch.Generator().manual_seed(11)
+    vote = (torch.rand(rows, n, generator=g) ** 4).cuda()
+    before = vote.clone()
+    first = sk.snapkv_pool_topk(vote, kernel, PT[ptype], ksel)
+    torch.cuda.synchronize()
+    assert torch.equal(vote, before)
+    again = sk.snapkv_pool_topk(vote, kernel, PT[ptype], ksel)
+    assert torch.equal(first, again)
+    assert torch.equal(vote, before)
+
+
 # ------------------------------------------------------------------ gather
 @pytest.mark.parametrize("B,Hq,Hkv,L,d,W,ksel", [
     (1, 4, 4, 1024, 64, 32, 224),
